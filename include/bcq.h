@@ -1,0 +1,163 @@
+/*
+ * bcq.h -- C ABI of the B200 (sm_100a) library for AlphaTuning's binary-coding-quantized
+ * (BCQ) linear layer.
+ *
+ * The layer stores a weight matrix W (d_out x d_in; the paper's h_out x h_in) as
+ *     W ~= sum_{i=1..q} diag(alpha_i) * B_i ,   B_i in {-1,+1}^{d_out x d_in}        (Eq. 1)
+ * with q bit-planes and fp32 scales alpha that are shared by groups of g consecutive weights
+ * of a row (Section "BCQ Format"; group-wise extension in the Appendix paragraph
+ * "group-wise quantization"; g = d_in is the row-wise scheme of Eq. 1).
+ *
+ * Conventions common to every call
+ *   - All data pointers are DEVICE pointers on the current CUDA device unless a parameter is
+ *     documented as host memory.  The caller owns every buffer; the library never allocates or
+ *     frees device memory.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream);
+ *     no call synchronises.
+ *   - The return value is the only error channel.  Arguments are validated on the host before
+ *     anything is launched; on an error nothing has been enqueued.
+ *   - Kernels never trap.  Every wait inside a kernel is time-limited; if one expires the kernel
+ *     records it in a device flag (see bcq_device_timeout_flag) and returns.
+ *
+ * Container format of a quantized matrix, G = ceil(d_in / g):
+ *   bits  : uint32 [q][d_out][pitch],  pitch = bcq_pitch_words(d_in) = 4 * ceil(d_in / 128);
+ *           bit (k & 31) of word (k >> 5) of row (i, j) is 1  <=>  b_i[j,k] = +1;
+ *           padding bits (k >= d_in) are 0.  Rows are 16-byte aligned.
+ *   alpha : float  [q][d_out][G];  alpha[i][j][c] scales weights k in [c*g, min((c+1)*g, d_in)).
+ *
+ * Supported shapes: 1 <= q <= 8, 1 <= d_out, 1 <= d_in, and either g == d_in or
+ * (g % 32 == 0 and 32 <= g <= d_in).  Other (q, g) give BCQ_ERR_UNSUPPORTED.
+ * bf16 tensors (X, dY) must be 16-byte aligned with a row pitch that is a multiple of 8
+ * elements (BCQ_ERR_ALIGN otherwise).
+ */
+#ifndef BCQ_H_
+#define BCQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BCQ_OK = 0,
+    BCQ_ERR_NULL = -1,          /* a required pointer is NULL */
+    BCQ_ERR_SHAPE = -2,         /* a size or pitch is out of range */
+    BCQ_ERR_ALIGN = -3,         /* a pointer or pitch breaks the alignment rules above */
+    BCQ_ERR_UNSUPPORTED = -4,   /* valid BCQ problem, but outside what the kernels cover */
+    BCQ_ERR_WORKSPACE = -5,     /* ws_bytes smaller than bcq_workspace_bytes() */
+    BCQ_ERR_CUDA = -6,          /* a CUDA call failed; see bcq_last_cuda_error() */
+    BCQ_ERR_DEVICE_TIMEOUT = -7 /* a kernel gave up on a wait (bcq_device_timeout_flag) */
+} bcq_status;
+
+typedef enum { BCQ_F32 = 0, BCQ_BF16 = 1 } bcq_dtype;
+
+typedef enum {
+    BCQ_OP_QUANTIZE = 0,
+    BCQ_OP_FWD = 1,
+    BCQ_OP_DECODE = 2,
+    BCQ_OP_BWD_X = 3,
+    BCQ_OP_BWD_ALPHA = 4
+} bcq_op;
+
+/* ------------------------------------------------------------------ sizes (host only) */
+
+/* Row pitch of `bits` in 32-bit words: 4 * ceil(d_in / 128).  0 if d_in < 1. */
+size_t bcq_pitch_words(int d_in);
+/* Bytes of the `bits` buffer: q * d_out * pitch * 4. */
+size_t bcq_bits_bytes(int d_out, int d_in, int q);
+/* G = ceil(d_in / g).  0 if g < 1. */
+size_t bcq_num_groups(int d_in, int g);
+/* Number of floats in `alpha`: q * d_out * G. */
+size_t bcq_alpha_count(int d_out, int d_in, int q, int g);
+/* Size of the quantized layer the way Table 1 counts it, in BITS (one bit per plane and
+ * weight, 32 bits per scale): q*d_out*d_in + 32*q*d_out*G. */
+size_t bcq_payload_bits(int d_out, int d_in, int q, int g);
+/* Bytes of scratch (`ws`) that operation `op` needs for this shape and token count n
+ * (n is ignored for BCQ_OP_QUANTIZE).  May be 0.  The scratch holds partial sums between the
+ * main kernel and its reduction; its contents are undefined afterwards and it must not be
+ * shared by calls that may overlap on the GPU. */
+size_t bcq_workspace_bytes(int op, int d_out, int d_in, int q, int g, int n);
+
+/* ------------------------------------------------------------------ quantizer */
+
+/* Post-training BCQ of W, one independent problem per (row, group).
+ *
+ * alt_iters = 0: Greedy approximation (Appendix, Eq. ap:1-ap:3): r = w; for each plane
+ *   b_i = sign(r) with sign(0) = +1, alpha_i = mean|r| over the group, r -= alpha_i b_i.
+ * alt_iters = T > 0: Alternating method (Appendix, Eq. ap:4 and the paragraph after it):
+ *   starting from the greedy result, T rounds of [least-squares alpha for the current signs,
+ *   then every weight moves to the nearest of the 2^q levels sum_i +-alpha_i; among
+ *   equidistant levels the one with the largest code sum_i 2^i [b_i = +1] wins], followed by one
+ *   last least-squares fit.  A group whose planes make B^T B singular keeps its previous
+ *   alpha in that round.
+ * Sums, residuals and the q x q solve are carried in fp64; every alpha is rounded to fp32 as
+ * soon as it is computed and the rounded value is used from then on.
+ *
+ *   W      in : float [d_out][ldw], ldw >= d_in
+ *   bits   out: container format above (padding bits are written as 0)
+ *   alpha  out: container format above
+ *   sq_err out: float64 [d_out][G], sum over the group of (w - w_hat)^2; may be NULL
+ * Group sizes up to 32768 are supported. */
+bcq_status bcq_quantize(int d_out, int d_in, int q, int g, const float* W, size_t ldw,
+                        int alt_iters, uint32_t* bits, float* alpha, double* sq_err,
+                        void* stream);
+
+/* W_hat[j][k] = sum_i alpha[i][j][k/g] * b_i[j,k]  (Eq. 1), fp32, W_hat: float [d_out][ldw]. */
+bcq_status bcq_dequantize(int d_out, int d_in, int q, int g, const uint32_t* bits,
+                          const float* alpha, float* W_hat, size_t ldw, void* stream);
+
+/* ------------------------------------------------------------------ linear layer */
+
+/* Forward (Eq. 2), computed from the packed planes without materialising W in memory:
+ *     Y[t][j] = sum_i sum_c alpha[i][j][c] * sum_{k in group c} X[t][k] * b_i[j,k]  (+ bias[j])
+ *   X    in : bf16 [n][ldx]
+ *   bias in : float [d_out] or NULL (the frozen bias of the layer)
+ *   Y    out: y_dtype [n][ldy], ldy >= d_out
+ *   ws      : scratch of bcq_workspace_bytes(BCQ_OP_FWD, ...) bytes, 16-byte aligned (NULL if 0)
+ * Products are bf16 x bf16 accumulated in fp32; the scaled weight sum_i alpha_i b_i enters
+ * the tensor core rounded to bf16. */
+bcq_status bcq_linear_fwd(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                          const uint32_t* bits, const float* alpha, const float* bias, void* Y,
+                          size_t ldy, int y_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/* Same computation for the decode regime, 1 <= n <= 16 tokens, where the cost is streaming
+ * the packed planes from memory once (Section "Inference Speed").  Workspace op is
+ * BCQ_OP_DECODE.  n > 16 gives BCQ_ERR_SHAPE. */
+bcq_status bcq_linear_decode(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                             const uint32_t* bits, const float* alpha, const float* bias,
+                             void* Y, size_t ldy, int y_dtype, void* ws, size_t ws_bytes,
+                             void* stream);
+
+/* Input gradient (Eq. 3):  dX[t][k] = sum_j dY[t][j] * W_hat[j][k],  W_hat as in Eq. 1.
+ *   dY in : bf16 [n][lddy];   dX out: dx_dtype [n][lddx], lddx >= d_in. */
+bcq_status bcq_linear_bwd_x(int d_out, int d_in, int q, int g, int n, const void* dY, size_t lddy,
+                            const uint32_t* bits, const float* alpha, void* dX, size_t lddx,
+                            int dx_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/* Scale gradient (Eq. 4, read as the chain rule through Eq. 1 and Eq. 2):
+ *     dalpha[i][j][c] (+)= scale * sum_{k in group c} b_i[j,k] * sum_t dY[t][j] * X[t][k]
+ * for every plane i whose bit is set in plane_mask; entries of other planes are not touched.
+ * scale = 1 gives the gradient; scale = 1/g gives the paper's stabilised update.  The
+ * d_out x d_in product dY^T X only ever exists tile by tile on chip.
+ *   accumulate: 0 overwrites dalpha, 1 adds to it.
+ *   dalpha out: float [q][d_out][G]. */
+bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, int n, const void* dY,
+                                size_t lddy, const void* X, size_t ldx, const uint32_t* bits,
+                                uint32_t plane_mask, float scale, int accumulate, float* dalpha,
+                                void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------ status */
+
+const char* bcq_status_string(int status);
+/* cudaError_t value of the last CUDA failure seen by this library on the calling thread. */
+int bcq_last_cuda_error(void);
+/* Reads (and with reset != 0 clears) the device-side flag that kernels set when a bounded wait
+ * expired.  Synchronises the device.  *flag_out = 0 means no kernel has given up. */
+bcq_status bcq_device_timeout_flag(int* flag_out /* host */, int reset);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCQ_H_ */

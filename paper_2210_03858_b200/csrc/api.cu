@@ -1,0 +1,50 @@
+// Host-only entry points: size helpers of the container format, status strings, error state.
+#include "common.h"
+
+namespace bcq {
+static thread_local int t_last_cuda_error = 0;
+void set_last_cuda_error(int e) { t_last_cuda_error = e; }
+}  // namespace bcq
+
+extern "C" size_t bcq_pitch_words(int d_in) {
+    return d_in < 1 ? 0 : 4 * (((size_t)d_in + 127) / 128);
+}
+
+extern "C" size_t bcq_bits_bytes(int d_out, int d_in, int q) {
+    if (d_out < 1 || q < 1) return 0;
+    return (size_t)q * (size_t)d_out * bcq_pitch_words(d_in) * sizeof(uint32_t);
+}
+
+extern "C" size_t bcq_num_groups(int d_in, int g) {
+    return (g < 1 || d_in < 1) ? 0 : ((size_t)d_in + (size_t)g - 1) / (size_t)g;
+}
+
+extern "C" size_t bcq_alpha_count(int d_out, int d_in, int q, int g) {
+    if (d_out < 1 || q < 1) return 0;
+    return (size_t)q * (size_t)d_out * bcq_num_groups(d_in, g);
+}
+
+extern "C" size_t bcq_payload_bits(int d_out, int d_in, int q, int g) {
+    if (d_out < 1 || d_in < 1 || q < 1 || g < 1) return 0;
+    return (size_t)q * (size_t)d_out * (size_t)d_in + 32 * bcq_alpha_count(d_out, d_in, q, g);
+}
+
+extern "C" const char* bcq_status_string(int status) {
+    switch (status) {
+        case BCQ_OK: return "ok";
+        case BCQ_ERR_NULL: return "a required pointer is NULL";
+        case BCQ_ERR_SHAPE: return "a size or pitch is out of range";
+        case BCQ_ERR_ALIGN: return "a pointer or pitch is not aligned as required";
+        case BCQ_ERR_UNSUPPORTED: return "shape not covered by the kernels (q > 8, or g neither d_in nor a multiple of 32)";
+        case BCQ_ERR_WORKSPACE: return "workspace smaller than bcq_workspace_bytes()";
+        case BCQ_ERR_CUDA: return "a CUDA call failed (see bcq_last_cuda_error)";
+        case BCQ_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int bcq_last_cuda_error(void) { return bcq::t_last_cuda_error; }
+
+extern "C" bcq_status bcq_device_timeout_flag(int* flag_out, int reset) {
+    return bcq::gemm_timeout_flag(flag_out, reset);
+}

@@ -1,0 +1,43 @@
+// Host-side helpers shared by the translation units of the library (no device code here).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/bcq.h"
+
+#define BCQ_MAX_Q 8
+#define BCQ_MAX_QUANT_G 32768
+
+namespace bcq {
+
+// cudaError_t of the last failing CUDA call on this thread (read by bcq_last_cuda_error()).
+void set_last_cuda_error(int e);
+
+inline bcq_status cuda_fail(cudaError_t e) {
+    set_last_cuda_error((int)e);
+    return BCQ_ERR_CUDA;
+}
+
+#define BCQ_CUDA_TRY(expr)                                  \
+    do {                                                    \
+        cudaError_t e__ = (expr);                           \
+        if (e__ != cudaSuccess) return bcq::cuda_fail(e__); \
+    } while (0)
+
+// Shape rules shared by every entry point (see include/bcq.h).
+inline bcq_status check_shape(int d_out, int d_in, int q, int g) {
+    if (d_out < 1 || d_in < 1 || q < 1 || g < 1 || g > d_in) return BCQ_ERR_SHAPE;
+    if (q > BCQ_MAX_Q) return BCQ_ERR_UNSUPPORTED;
+    if (g != d_in && (g % 32) != 0) return BCQ_ERR_UNSUPPORTED;
+    return BCQ_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Reads / clears the device flag set by kernels whose bounded waits expired.
+bcq_status gemm_timeout_flag(int* flag_out, int reset);
+
+}  // namespace bcq

@@ -1,0 +1,238 @@
+"""GPU parity: every CUDA entry point, called through the C-ABI binding, against the fp64 CPU
+oracle on the same seeded inputs.
+
+Tolerances:
+  * packed bits: bit-exact, except in groups the oracle flags as near-ties (decision margin
+    below 2^-20 of mean|w|), where rounding order may legitimately flip a bit;
+  * quantizer alpha: |a - a_ref| <= 1e-5 * max(|a_ref|, mean|w_group|);
+  * fp32 outputs of fwd / dX / dalpha: max|out - ref| / max|ref| <= 2e-3 (bf16 operands, fp32
+    accumulation, the scaled weight rounded once to bf16);
+  * bf16 outputs: the same bound plus one bf16 rounding (2^-8 relative).
+"""
+import numpy as np
+import pytest
+
+import oracle
+import paper_2210_03858_b200 as bcq
+from paper_2210_03858_b200 import build as bcq_build
+from paper_2210_03858_b200 import synth
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+TOL = 2e-3
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    bcq_build.build_library()
+    assert torch.cuda.is_available()
+    yield
+    assert bcq.device_timeout_flag() == 0, "a kernel reported an expired wait"
+
+
+def dev_bf16(a_u16):
+    return torch.from_numpy(a_u16.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def dev_bits(bits_u32):
+    return torch.from_numpy(bits_u32.view(np.int32)).cuda()
+
+
+def host_bits(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def rel_err(out, ref):
+    return float(np.abs(out.astype(np.float64) - ref).max() / np.abs(ref).max())
+
+
+def make_case(seed, n, d_in, d_out, q, g, alt=0, outliers=0.0):
+    key = (100, seed, 0)
+    W = synth.weights(d_out, d_in, key, outlier_frac=outliers)
+    X = synth.activations(n, d_in, key, synth.ROLE_X)
+    dY = synth.activations(n, d_out, key, synth.ROLE_DY)
+    bits, alpha, sq_err, margin = oracle.quantize(W, q, g, alt_iters=alt)
+    return W, X, dY, bits, alpha, sq_err, margin
+
+
+# --------------------------------------------------------------------------- quantizer
+
+QUANT_CASES = [
+    # d_out, d_in, q, g, alt, outliers
+    (64, 128, 3, 128, 0, 0.0),
+    (37, 1000, 3, 1000, 0, 0.0),      # row-wise, d_in not a multiple of 32
+    (50, 1600, 4, 128, 0, 0.0),       # ragged last group (64)
+    (24, 1024, 1, 32, 0, 0.0),
+    (9, 4096, 2, 4096, 0, 0.0),       # CTA-wide teams
+    (3, 20480, 2, 20480, 0, 0.0),
+    (5, 8192, 8, 2048, 0, 0.0),
+    (40, 512, 2, 128, 5, 1e-3),
+    (40, 512, 3, 128, 5, 1e-3),
+    (40, 640, 4, 128, 5, 1e-3),
+    (16, 1024, 3, 1024, 3, 0.0),
+    (6, 2304, 4, 2304, 2, 0.0),
+    (12, 200, 5, 200, 1, 0.0),
+]
+
+
+@pytest.mark.parametrize("d_out,d_in,q,g,alt,outl", QUANT_CASES)
+def test_quantize_matches_oracle(d_out, d_in, q, g, alt, outl):
+    W, _, _, bits_ref, alpha_ref, sq_ref, margin = make_case(d_in + q, 1, d_in, d_out, q, g, alt, outl)
+    bits, alpha, sq_err = bcq.quantize(torch.from_numpy(W).cuda(), q, g, alt, want_sq_err=True)
+    torch.cuda.synchronize()
+    bits, alpha, sq_err = host_bits(bits), alpha.cpu().numpy(), sq_err.cpu().numpy()
+    G = oracle.num_groups(d_in, g)
+    # padding bits are zero
+    total = bits.shape[2] * 32
+    kk = np.arange(d_in, total)
+    if kk.size:
+        assert not ((bits[:, :, kk >> 5] >> (kk & 31).astype(np.uint32)) & 1).any()
+    flagged = margin < 2.0 ** -20
+    diff_words = bits != bits_ref
+    if diff_words.any():
+        # every differing bit must sit in a flagged group
+        k = np.arange(d_in)
+        dbit = ((bits ^ bits_ref)[:, :, k >> 5] >> (k & 31).astype(np.uint32)) & 1
+        for c in range(G):
+            bad = dbit[:, :, c * g:(c + 1) * g].any(axis=(0, 2))
+            assert not (bad & ~flagged[:, c]).any(), "bits differ in a group that is not a near-tie"
+    same = ~np.stack([(bits != bits_ref)[:, :, (c * g) >> 5:((min((c + 1) * g, d_in) + 31) >> 5)].any(axis=(0, 2))
+                      for c in range(G)], axis=1)
+    assert same.mean() > 0.999
+    mean_abs = np.stack([np.abs(W[:, c * g:(c + 1) * g]).mean(axis=1) for c in range(G)], axis=1)
+    tol = 1e-5 * np.maximum(np.abs(alpha_ref), mean_abs[None])
+    ok = np.abs(alpha - alpha_ref) <= tol
+    assert ok[:, same].all()
+    np.testing.assert_allclose(sq_err[same], sq_ref[same], rtol=1e-6, atol=1e-18)
+
+
+def test_quantize_strided_input_and_determinism():
+    W = synth.weights(48, 384, (101, 0, 0))
+    Wp = np.zeros((48, 400), dtype=np.float32)
+    Wp[:, :384] = W
+    ref_bits, ref_alpha, _, _ = oracle.quantize(W, 3, 128)
+    Wd = torch.from_numpy(Wp).cuda()[:, :384]
+    b1, a1, _ = bcq.quantize(Wd, 3, 128)
+    b2, a2, _ = bcq.quantize(Wd, 3, 128)
+    torch.cuda.synchronize()
+    assert torch.equal(b1, b2) and torch.equal(a1, a2)
+    np.testing.assert_array_equal(host_bits(b1), ref_bits)
+    np.testing.assert_array_equal(a1.cpu().numpy(), ref_alpha)
+
+
+def test_dequantize_matches_oracle():
+    for (d_out, d_in, q, g) in ((33, 1000, 3, 1000), (20, 1600, 4, 128), (7, 96, 2, 32)):
+        _, _, _, bits, alpha, _, _ = make_case(7, 1, d_in, d_out, q, g)
+        out = bcq.dequantize(dev_bits(bits), torch.from_numpy(alpha).cuda(), d_in, g).cpu().numpy()
+        ref = oracle.dequantize(bits, alpha, d_in, g)
+        np.testing.assert_allclose(out, ref, rtol=1e-6, atol=1e-9)
+
+
+# --------------------------------------------------------------------------- linear layer
+
+LINEAR_CASES = [
+    # n, d_in, d_out, q, g
+    (512, 1024, 1024, 3, 1024),    # the single-layer workload: several tiles, row-wise
+    (300, 1000, 200, 4, 1000),     # ragged everywhere, row-wise with d_in % 32 != 0
+    (257, 1600, 330, 4, 128),      # ragged last group, partial tiles in every dimension
+    (64, 256, 128, 1, 32),         # smallest group size
+    (130, 320, 384, 2, 96),        # groups not aligned to the tile widths
+    (1100, 512, 640, 3, 256),      # more token tiles than one wave of a small grid
+    (96, 2048, 256, 8, 512),       # q = 8
+]
+
+
+def _upload(X, dY, bits, alpha):
+    return dev_bf16(X), dev_bf16(dY), dev_bits(bits), torch.from_numpy(alpha).cuda()
+
+
+@pytest.mark.parametrize("n,d_in,d_out,q,g", LINEAR_CASES)
+def test_fwd_matches_oracle(n, d_in, d_out, q, g):
+    _, X, dY, bits, alpha, _, _ = make_case(n, n, d_in, d_out, q, g)
+    Xd, _, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    Y = bcq.linear_fwd(Xd, bd, ad, d_in, g)
+    Y2 = bcq.linear_fwd(Xd, bd, ad, d_in, g)
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2), "two runs differ"
+    assert rel_err(Y.cpu().numpy(), ref) <= TOL
+    # bias and bf16 output
+    bias = synth.bias(d_out, (100, n, 0))
+    Yb = bcq.linear_fwd(Xd, bd, ad, d_in, g, bias=torch.from_numpy(bias).cuda(),
+                        out_dtype=torch.bfloat16)
+    refb = ref + bias.astype(np.float64)
+    assert rel_err(Yb.float().cpu().numpy(), refb) <= TOL + 2.0 ** -8
+
+
+@pytest.mark.parametrize("n,d_in,d_out,q,g", LINEAR_CASES)
+def test_bwd_x_matches_oracle(n, d_in, d_out, q, g):
+    _, X, dY, bits, alpha, _, _ = make_case(n, n, d_in, d_out, q, g)
+    _, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.bwd_x(dY, bits, alpha, d_in, g)
+    dX = bcq.linear_bwd_x(dYd, bd, ad, d_in, g)
+    dX2 = bcq.linear_bwd_x(dYd, bd, ad, d_in, g)
+    torch.cuda.synchronize()
+    assert torch.equal(dX, dX2)
+    assert rel_err(dX.cpu().numpy(), ref) <= TOL
+    dXb = bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=torch.bfloat16)
+    assert rel_err(dXb.float().cpu().numpy(), ref) <= TOL + 2.0 ** -8
+
+
+@pytest.mark.parametrize("n,d_in,d_out,q,g", LINEAR_CASES)
+def test_bwd_alpha_matches_oracle(n, d_in, d_out, q, g):
+    _, X, dY, bits, alpha, _, _ = make_case(n, n, d_in, d_out, q, g)
+    Xd, dYd, bd, _ = _upload(X, dY, bits, alpha)
+    ref = oracle.bwd_alpha(dY, X, bits, d_in, g)
+    dA = bcq.linear_bwd_alpha(dYd, Xd, bd, d_in, g)
+    dA2 = bcq.linear_bwd_alpha(dYd, Xd, bd, d_in, g)
+    torch.cuda.synchronize()
+    assert torch.equal(dA, dA2)
+    assert rel_err(dA.cpu().numpy(), ref) <= TOL
+    # alpha_1 only, the paper's 1/g scale, accumulate on top of existing values
+    out = torch.full_like(dA, 3.0)
+    bcq.linear_bwd_alpha(dYd, Xd, bd, d_in, g, plane_mask=1, scale=1.0 / g, accumulate=True, out=out)
+    o = out.cpu().numpy()
+    assert (o[1:] == 3.0).all()
+    assert np.abs(o[0] - 3.0 - ref[0] / g).max() <= TOL * np.abs(ref[0] / g).max() + 1e-6
+
+
+@pytest.mark.parametrize("n", [1, 4, 16, 5])
+@pytest.mark.parametrize("d_in,d_out,q,g", [(4096, 1536, 3, 128), (1024, 520, 4, 128), (2048, 256, 3, 2048)])
+def test_decode_matches_oracle(n, d_in, d_out, q, g):
+    _, X, dY, bits, alpha, _, _ = make_case(n + d_out, n, d_in, d_out, q, g)
+    Xd, _, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    Y = bcq.linear_decode(Xd, bd, ad, d_in, g)
+    Y2 = bcq.linear_decode(Xd, bd, ad, d_in, g)
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2)
+    assert rel_err(Y.cpu().numpy(), ref) <= TOL
+
+
+def test_strided_activations_and_outputs():
+    n, d_in, d_out, q, g = 70, 256, 192, 3, 128
+    _, X, dY, bits, alpha, _, _ = make_case(3, n, d_in, d_out, q, g)
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    Xp = torch.zeros((n, d_in + 8), dtype=torch.bfloat16, device="cuda")
+    Xp[:, :d_in] = Xd
+    Yp = torch.full((n, d_out + 5), -7.0, dtype=torch.float32, device="cuda")
+    bcq.linear_fwd(Xp[:, :d_in], bd, ad, d_in, g, out=Yp[:, :d_out])
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    assert rel_err(Yp[:, :d_out].cpu().numpy(), ref) <= TOL
+    assert (Yp[:, d_out:] == -7.0).all()       # nothing written past the row
+
+
+def test_quantize_then_layer_end_to_end():
+    # the whole path on device: W -> (bits, alpha) -> fwd, dX, dalpha, all against the oracle
+    n, d_in, d_out, q, g = 256, 512, 384, 3, 128
+    W, X, dY, bits_ref, alpha_ref, _, _ = make_case(11, n, d_in, d_out, q, g)
+    bits, alpha, _ = bcq.quantize(torch.from_numpy(W).cuda(), q, g)
+    np.testing.assert_array_equal(host_bits(bits), bits_ref)
+    Xd, dYd = dev_bf16(X), dev_bf16(dY)
+    assert rel_err(bcq.linear_fwd(Xd, bits, alpha, d_in, g).cpu().numpy(),
+                   oracle.fwd(X, bits_ref, alpha_ref, d_in, g)) <= TOL
+    assert rel_err(bcq.linear_bwd_x(dYd, bits, alpha, d_in, g).cpu().numpy(),
+                   oracle.bwd_x(dY, bits_ref, alpha_ref, d_in, g)) <= TOL
+    assert rel_err(bcq.linear_bwd_alpha(dYd, Xd, bits, d_in, g).cpu().numpy(),
+                   oracle.bwd_alpha(dY, X, bits_ref, d_in, g)) <= TOL
