@@ -135,7 +135,7 @@ LINEAR_CASES = [
     # n, d_in, d_out, q, g
     (512, 1024, 1024, 3, 1024),    # the single-layer workload: several tiles, row-wise
     (300, 1000, 200, 4, 1000),     # ragged everywhere, row-wise with d_in % 32 != 0
-    (257, 1600, 330, 4, 128),      # ragged last group, partial tiles in every dimension
+    (257, 1600, 336, 4, 128),      # ragged last group, partial tiles in every dimension
     (64, 256, 128, 1, 32),         # smallest group size
     (130, 320, 384, 2, 96),        # groups not aligned to the tile widths
     (1100, 512, 640, 3, 256),      # more token tiles than one wave of a small grid
