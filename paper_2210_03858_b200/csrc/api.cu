@@ -1,5 +1,5 @@
 // Host-only entry points: size helpers of the container format, status strings, error state.
-#include "common.h"
+#include "gemm_common.cuh"
 
 namespace bcq {
 static thread_local int t_last_cuda_error = 0;
@@ -46,5 +46,25 @@ extern "C" const char* bcq_status_string(int status) {
 extern "C" int bcq_last_cuda_error(void) { return bcq::t_last_cuda_error; }
 
 extern "C" bcq_status bcq_device_timeout_flag(int* flag_out, int reset) {
-    return bcq::gemm_timeout_flag(flag_out, reset);
+    if (flag_out == nullptr) return BCQ_ERR_NULL;
+    BCQ_CUDA_TRY(cudaDeviceSynchronize());
+    int a = 0, b = 0;
+    bcq_status st = bcq::expand_timeout_flag(&a, reset);
+    if (st != BCQ_OK) return st;
+    st = bcq::dalpha_timeout_flag(&b, reset);
+    if (st != BCQ_OK) return st;
+    *flag_out = a != 0 ? a : b;
+    return BCQ_OK;
+}
+
+extern "C" size_t bcq_workspace_bytes(int op, int d_out, int d_in, int q, int g, int n) {
+    if (bcq::check_shape(d_out, d_in, q, g) != BCQ_OK) return 0;
+    if (op != BCQ_OP_QUANTIZE && n < 1) return 0;
+    switch (op) {
+        case BCQ_OP_FWD: return bcq::fwd_workspace_bytes(d_out, d_in, q, g, n);
+        case BCQ_OP_DECODE: return n > 16 ? 0 : bcq::decode_workspace_bytes(d_out, d_in, q, g, n);
+        case BCQ_OP_BWD_X: return bcq::bwd_x_workspace_bytes(d_out, d_in, q, g, n);
+        case BCQ_OP_BWD_ALPHA: return bcq::bwd_alpha_workspace_bytes(d_out, d_in, q, g, n);
+        default: return 0;
+    }
 }

@@ -37,7 +37,4 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// Reads / clears the device flag set by kernels whose bounded waits expired.
-bcq_status gemm_timeout_flag(int* flag_out, int reset);
-
 }  // namespace bcq

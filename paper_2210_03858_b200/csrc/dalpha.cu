@@ -1,0 +1,361 @@
+// Scale gradient of the BCQ linear layer (Eq. 4):
+//     dalpha_i[j, c] = scale * sum_{k in group c} b_i[j,k] * (dY^T X)[j,k].
+//
+// D[j, k] = sum_t dY[t, j] X[t, k] is a 128 x TN x 64 UMMA tile product with both operands
+// MN-major (tokens are the K index; dY and X rows are contiguous in j and k), loaded by TMA in
+// 64 x 64 boxes.  The epilogue never writes D: thread = (row j, half of the tile's columns) reads
+// its accumulator row from tensor memory 32 columns at a time, applies the signs of every
+// requested plane from one 32-bit word of the packed planes, and sums per group.  Partial sums
+// (one per split over tokens, column sub-tile and group piece) go to the workspace and a second
+// kernel adds them in a fixed order, so the result does not depend on scheduling.
+#include "gemm_common.cuh"
+
+namespace {
+
+using namespace bcq;
+
+__device__ int g_timeout_flag = 0;
+
+struct DalphaParams {
+    int d_out, d_in, q, g, G, pitch, n;
+    int num_kb;          // K blocks of 64 tokens
+    int kb_per_split;
+    int splits;
+    int n_subtiles;      // column sub-tiles of width TN/2 over d_in
+    int slots;           // partial slots per sub-tile
+    uint32_t plane_mask;
+    const uint32_t* bits;
+    float* partial;      // [splits][n_subtiles][q][slots][d_out]
+};
+
+
+// ------------------------------------------------------------------------------------------
+// dalpha: D[j, k] = sum_t dY[t, j] X[t, k], sign-weighted group sums in the epilogue
+// ------------------------------------------------------------------------------------------
+
+template <int TN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
+              const DalphaParams p) {
+    constexpr uint32_t kBBytes = TN * kBlockK * 2;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kIdesc = ptx::make_idesc_bf16(kBlockM, TN, 1, 1);
+    constexpr int HN = TN / 2;
+    constexpr int NCH = HN / 32;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t ctl_base = smem_base + STAGES * kStageBytes;
+    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes;
+
+    Ctl ctl;
+    ctl.full = ctl_base;
+    ctl.aready = 0;
+    ctl.empty = ctl_base + 8 * STAGES;
+    ctl.accum = ctl_base + 16 * STAGES;
+    ctl.spare = ctl.accum + 8;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 16 * STAGES + 16);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 16 * STAGES + 20);
+    ctl.device_flag = &g_timeout_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int j0 = blockIdx.x * kBlockM;
+    const int k0 = blockIdx.y * TN;
+    const int kb_begin = blockIdx.z * p.kb_per_split;
+    const int kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+    const int iters = kb_end - kb_begin;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(ctl.full + 8 * s, 1);
+            ptx::mbar_init(ctl.empty + 8 * s, 1);
+        }
+        ptx::mbar_init(ctl.accum, 1);
+        ptx::mbar_init(ctl.spare, 1);
+        *ctl.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_dy);
+        ptx::prefetch_tmap(&tmap_x);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), TmemCols<TN>::value);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            bool ok = true;
+            int issued = 0;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 11);
+                if (!ok) break;
+                const uint32_t sa = smem_base + s * kStageBytes;
+                const int tok = (kb_begin + it) * kBlockK;
+                ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kStageBytes);
+                // A: two blocks of 64 rows j (inner) x 64 tokens; B: TN/64 blocks of 64 k x 64 tokens
+                ptx::tma_load_2d(sa, &tmap_dy, j0, tok, ctl.full + 8 * s);
+                ptx::tma_load_2d(sa + 8192, &tmap_dy, j0 + 64, tok, ctl.full + 8 * s);
+#pragma unroll
+                for (int b = 0; b < TN / 64; ++b)
+                    ptx::tma_load_2d(sa + kABytes + b * 8192, &tmap_x, k0 + b * 64, tok, ctl.full + 8 * s);
+                issued = it + 1;
+            }
+            if (!ok) {
+                for (int it = max(0, issued - STAGES); it < issued; ++it)
+                    wait_bar(ctl.full + 8 * (it % STAGES), (it / STAGES) & 1, ctl, 12);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 13);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t sa = smem_base + s * kStageBytes;
+                const uint32_t sb = sa + kABytes;
+#pragma unroll
+                for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                    const uint64_t da = ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
+                    const uint64_t db = ptx::make_smem_desc(sb + kk * 2048, 8192, 1024);
+                    ptx::umma_bf16(tmem_base, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::umma_commit(ctl.empty + 8 * s);
+            }
+            if (ok) {
+                ptx::umma_commit(ctl.accum);
+            } else {
+                ptx::umma_commit(ctl.spare);
+                wait_bar(ctl.spare, 0, ctl, 15);
+            }
+        }
+    } else {
+        // ---------------- epilogue: thread = (row j, HN columns of the tile)
+        const int quarter = warp & 3;
+        const int half = (warp - kWorkerWarp0) >> 2;
+        const int j = j0 + quarter * 32 + lane;
+        const bool j_ok = j < p.d_out;
+        const int kbase = k0 + half * HN;
+        const int subtile = blockIdx.y * 2 + half;
+        const long long plane_words = (long long)p.d_out * p.pitch;
+
+        // the sign words do not depend on the accumulator: fetch them while the main loop runs
+        uint32_t nw[NCH][BCQ_MAX_Q];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) {
+            const int kw = (kbase >> 5) + ch;
+#pragma unroll
+            for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                const bool act = (i < p.q) && ((p.plane_mask >> i) & 1u) && j_ok && (kw < p.pitch);
+                nw[ch][i] = act ? ~__ldg(p.bits + i * plane_words + (long long)j * p.pitch + kw) : 0u;
+            }
+        }
+
+        bool ok = wait_bar(ctl.accum, 0, ctl, 16);
+        if (ok && kbase < p.d_in) {
+            ptx::tc_fence_after_sync();
+            const int c_first = min(kbase / p.g, p.G - 1);
+            float acc[BCQ_MAX_Q];
+#pragma unroll
+            for (int i = 0; i < BCQ_MAX_Q; ++i) acc[i] = 0.0f;
+            int cur_c = c_first;
+            auto flush = [&](int c) {
+                if (!j_ok) return;
+                const int slot = c - c_first;
+#pragma unroll
+                for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                    if (i < p.q && ((p.plane_mask >> i) & 1u)) {
+                        const long long idx =
+                            ((((long long)blockIdx.z * p.n_subtiles + subtile) * p.q + i) * p.slots + slot) *
+                                p.d_out + j;
+                        p.partial[idx] = acc[i];
+                    }
+                }
+            };
+#pragma unroll
+            for (int ch = 0; ch < NCH; ++ch) {
+                const int kg = kbase + ch * 32;
+                if (kg < p.d_in) {  // uniform in the warp
+                    const int c = min(kg / p.g, p.G - 1);
+                    if (c != cur_c) {
+                        flush(cur_c);
+                        cur_c = c;
+#pragma unroll
+                        for (int i = 0; i < BCQ_MAX_Q; ++i) acc[i] = 0.0f;
+                    }
+                    uint32_t v[32];
+                    ptx::tmem_ld_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) +
+                                         (uint32_t)(half * HN + ch * 32), v);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                        if (i < p.q && ((p.plane_mask >> i) & 1u)) {
+                            const uint32_t w = nw[ch][i];
+                            float s = 0.0f;
+#pragma unroll
+                            for (int b = 0; b < 32; ++b)
+                                s += __uint_as_float(v[b] ^ ((w << (31 - b)) & 0x80000000u));
+                            acc[i] += s;
+                        }
+                    }
+                }
+            }
+            flush(cur_c);
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TmemCols<TN>::value);
+    }
+}
+
+// dalpha[i][j][c] (+)= scale * sum over splits and over the sub-tiles that meet group c.
+__global__ void dalpha_reduce_kernel(int d_out, int d_in, int q, int g, int G, int HN, int splits,
+                                     int n_subtiles, int slots, uint32_t plane_mask, float scale,
+                                     int accumulate, const float* __restrict__ partial,
+                                     float* __restrict__ dalpha) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)q * G * d_out;
+    if (idx >= total) return;
+    const int j = (int)(idx % d_out);
+    const long long r = idx / d_out;
+    const int c = (int)(r % G);
+    const int i = (int)(r / G);
+    if (!((plane_mask >> i) & 1u)) return;
+    const int k_lo = c * g;
+    const int k_hi = min(k_lo + g, d_in) - 1;
+    float s = 0.0f;
+    for (int z = 0; z < splits; ++z)
+        for (int st = k_lo / HN; st <= k_hi / HN; ++st) {
+            const int slot = c - min((st * HN) / g, G - 1);
+            s += __ldg(partial + ((((long long)z * n_subtiles + st) * q + i) * slots + slot) * d_out + j);
+        }
+    float* dst = dalpha + ((long long)i * d_out + j) * G + c;
+    *dst = accumulate ? (*dst + scale * s) : (scale * s);
+}
+
+struct DalphaPlan {
+    int TN, HN, splits, kb_per_split, num_kb, m_tiles, n_tiles, n_subtiles, slots;
+};
+
+DalphaPlan plan_dalpha(int d_out, int d_in, int g, int n) {
+    DalphaPlan pl;
+    const int sms = sm_count();
+    pl.m_tiles = ceil_div(d_out, kBlockM);
+    pl.num_kb = ceil_div(n, kBlockK);
+    pl.TN = 256;
+    if (d_in <= 128 || pl.m_tiles * ceil_div(d_in, 256) < sms) pl.TN = 128;
+    pl.HN = pl.TN / 2;
+    pl.n_tiles = ceil_div(d_in, pl.TN);
+    pl.n_subtiles = pl.n_tiles * 2;
+    if (g % pl.HN == 0) pl.slots = 1;
+    else if (pl.HN % g == 0) pl.slots = pl.HN / g;
+    else pl.slots = pl.HN / g + 2;
+    const int tiles = pl.m_tiles * pl.n_tiles;
+    int splits = sms / tiles;
+    if (splits < 1) splits = 1;
+    const int max_splits = (pl.num_kb + 3) / 4;
+    if (splits > max_splits) splits = max_splits;
+    if (splits > 32) splits = 32;
+    pl.kb_per_split = ceil_div(pl.num_kb, splits);
+    pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
+    return pl;
+}
+
+
+template <int TN>
+constexpr int stages_for() {
+    return TN == 256 ? 4 : 6;
+}
+
+template <int TN>
+constexpr size_t smem_for() {
+    return (size_t)stages_for<TN>() * (kABytes + TN * kBlockK * 2) + 1024 + 256;
+}
+
+size_t dalpha_ws_bytes(const DalphaPlan& pl, int d_out, int q) {
+    return (size_t)pl.splits * pl.n_subtiles * q * pl.slots * d_out * sizeof(float);
+}
+
+}  // namespace
+
+namespace bcq {
+bcq_status dalpha_timeout_flag(int* flag_out, int reset) {
+    int v = 0;
+    BCQ_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_timeout_flag, sizeof(int)));
+    *flag_out = v;
+    if (reset && v != 0) {
+        const int zero = 0;
+        BCQ_CUDA_TRY(cudaMemcpyToSymbol(g_timeout_flag, &zero, sizeof(int)));
+    }
+    return BCQ_OK;
+}
+
+size_t bwd_alpha_workspace_bytes(int d_out, int d_in, int q, int g, int n) {
+    return dalpha_ws_bytes(plan_dalpha(d_out, d_in, g, n), d_out, q);
+}
+}  // namespace bcq
+
+extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, int n, const void* dY,
+                                           size_t lddy, const void* X, size_t ldx, const uint32_t* bits,
+                                           uint32_t plane_mask, float scale, int accumulate,
+                                           float* dalpha, void* ws, size_t ws_bytes, void* stream) {
+    bcq_status st = check_shape(d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1) return BCQ_ERR_SHAPE;
+    if (!bits || !dalpha) return BCQ_ERR_NULL;
+    if ((st = check_act(dY, lddy, d_out)) != BCQ_OK) return st;
+    if ((st = check_act(X, ldx, d_in)) != BCQ_OK) return st;
+    if (!aligned16(bits)) return BCQ_ERR_ALIGN;
+    plane_mask &= (1u << q) - 1u;
+    if (plane_mask == 0) return BCQ_OK;
+    const DalphaPlan pl = plan_dalpha(d_out, d_in, g, n);
+    const size_t need = dalpha_ws_bytes(pl, d_out, q);
+    if (ws == nullptr) return BCQ_ERR_NULL;
+    if (ws_bytes < need) return BCQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return BCQ_ERR_ALIGN;
+
+    CUtensorMap tm_dy, tm_x;
+    if ((st = make_tmap_16bit(&tm_dy, dY, 0, d_out, n, lddy, 64)) != BCQ_OK) return st;
+    if ((st = make_tmap_16bit(&tm_x, X, 0, d_in, n, ldx, 64)) != BCQ_OK) return st;
+    DalphaParams p;
+    p.d_out = d_out; p.d_in = d_in; p.q = q; p.g = g;
+    p.G = (int)bcq_num_groups(d_in, g);
+    p.pitch = (int)bcq_pitch_words(d_in);
+    p.n = n; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
+    p.n_subtiles = pl.n_subtiles; p.slots = pl.slots; p.plane_mask = plane_mask;
+    p.bits = bits; p.partial = reinterpret_cast<float*>(ws);
+    cudaStream_t s = (cudaStream_t)stream;
+    dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.n_tiles, (unsigned)pl.splits);
+    if (pl.TN == 256) {
+        auto kern = dalpha_kernel<256, stages_for<256>()>;
+        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem_for<256>()));
+        kern<<<grid, kThreads, smem_for<256>(), s>>>(tm_dy, tm_x, p);
+    } else {
+        auto kern = dalpha_kernel<128, stages_for<128>()>;
+        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)smem_for<128>()));
+        kern<<<grid, kThreads, smem_for<128>(), s>>>(tm_dy, tm_x, p);
+    }
+    BCQ_CUDA_TRY(cudaGetLastError());
+    const long long total = (long long)q * p.G * d_out;
+    dalpha_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+        d_out, d_in, q, g, p.G, pl.HN, pl.splits, pl.n_subtiles, pl.slots, plane_mask, scale, accumulate,
+        p.partial, dalpha);
+    BCQ_CUDA_TRY(cudaGetLastError());
+    return BCQ_OK;
+}

@@ -1,0 +1,1147 @@
+// Forward (Eq. 2), input gradient (Eq. 3) and decode kernels of the BCQ linear layer.
+//
+//   forward / decode   D[j, t] = sum_k  W_hat[j, k] * X[t, k]
+//   dX                 D[k, t] = sum_j  W_hat[j, k] * dY[t, j]
+//
+// W_hat = sum_i alpha_i b_i (Eq. 1) never exists in global memory: worker warps rebuild it tile by
+// tile from the packed planes, straight into the 128-byte-swizzled shared-memory operand layout of
+// tcgen05.mma (K-major for the forward, where j is the M index; MN-major for dX, where k is the M
+// index and one 128-byte line holds 64 consecutive k of one row j).  Accumulators live in tensor
+// memory (128 lanes x TN fp32 columns).
+//
+// Number format.  A scaled weight rounded to bf16 (8 significant bits) alone already costs about
+// 1.7e-3 relative error on the outputs, so both operands are fp16 (11 bits):
+//   * the scaled weight takes one of 2^q values per (row, group).  For q <= 4 the workers build
+//     a byte-wise lookup table of the fp16 levels in four registers and index it with PRMT: the
+//     selector nibbles are the plane bits of four weights, gathered with shifts and masks.  For
+//     q = 4 the table holds the eight levels with b_4 = +1; b_4 = -1 mirrors the index and flips
+//     the sign.  q > 4 falls back to fp32 sums of +-alpha_i.
+//   * activations are bf16 at the interface.  A short pre-pass writes them to the workspace as
+//     fp16, each token row multiplied by a power of two that brings its largest magnitude to
+//     2^14..2^15 (exact; undone in the epilogue), so neither large activations nor small
+//     gradients leave the fp16 range.  The same pre-pass finds max|alpha|, from which a power of
+//     two for the weights is derived.  Decode (<= 16 tokens) has no pre-pass: every CTA converts
+//     the X slice it needs itself and scales per (token, K-slice) and per weight row.
+//   * within every aligned run of 8 consecutive k the tile stores k in the order
+//     0,4,1,5,2,6,3,7 (that is what one PRMT pair produces).  For the forward the pre-pass writes
+//     the activations in the same order; for dX, where k indexes accumulator rows, the epilogue
+//     maps rows back.
+#include "gemm_common.cuh"
+
+namespace {
+
+using namespace bcq;
+
+__device__ int g_timeout_flag = 0;
+
+enum { MODE_FWD = 0, MODE_BWDX = 1 };
+enum { QM_LUT3 = 0, QM_LUT4 = 1, QM_GENERIC = 2 };
+constexpr int kPrefetch = 3;  // stages between the global loads of a task and its use
+
+// ------------------------------------------------------------------------------------------
+// small device helpers
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+    __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// 2^e as a float, e clamped to the normal range.
+__device__ __forceinline__ float pow2f(int e) {
+    e = max(-126, min(127, e));
+    return __uint_as_float((uint32_t)(e + 127) << 23);
+}
+
+// Exponent of a positive finite float given by its bits (0 for zero / subnormal input).
+__device__ __forceinline__ int exponent_of_bits(uint32_t fbits) {
+    const int be = (int)((fbits >> 23) & 0xFFu);
+    return be == 0 ? -127 : be - 127;
+}
+
+// Power of two that brings a magnitude with exponent `e` to [2^target, 2^(target+1)).
+__device__ __forceinline__ int shift_for(int e, int target) {
+    if (e <= -127 || e >= 128) return 0;  // zero, subnormal, inf or nan: leave alone
+    return max(-100, min(100, target - e));
+}
+
+// Byte-wise lookup table of eight fp16 levels: tl* low bytes, th* high bytes; *0 = levels 0..3.
+struct Lut {
+    uint32_t tl0, tl1, th0, th1;
+};
+
+// Level s (bit i of s set <=> plane i is +1) = base + sum_{i<3} (+-a_i).
+__device__ __forceinline__ Lut build_lut(float a0, float a1, float a2, float base) {
+    const float t0 = base - a0, t1 = base + a0;
+    const float u0 = t0 - a1, u1 = t1 - a1, u2 = t0 + a1, u3 = t1 + a1;
+    const uint32_t p0 = pack_half2(u0 - a2, u1 - a2);
+    const uint32_t p1 = pack_half2(u2 - a2, u3 - a2);
+    const uint32_t p2 = pack_half2(u0 + a2, u1 + a2);
+    const uint32_t p3 = pack_half2(u2 + a2, u3 + a2);
+    Lut t;
+    t.tl0 = prmt(p0, p1, 0x6420u);
+    t.th0 = prmt(p0, p1, 0x7531u);
+    t.tl1 = prmt(p2, p3, 0x6420u);
+    t.th1 = prmt(p2, p3, 0x7531u);
+    return t;
+}
+
+// 32 weights of one row from the plane words w0..w3 through the lookup table, stored as four
+// 16-byte chunks (slots chunk0..chunk0+3) of the 128-byte line at `line` (swizzle key lx).
+// Chunk cc holds weights 8cc..8cc+7 in the order 0,4,1,5,2,6,3,7.
+template <bool Q4>
+__device__ __forceinline__ void expand32_lut(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                             const Lut& t, uint32_t line, uint32_t lx, uint32_t chunk0) {
+    uint32_t x0 = w0, x1 = w1, x2 = w2, nf = 0u;
+    if (Q4) {
+        // b_4 = -1 (bit clear): value = -level[~index]
+        nf = ~w3;
+        x0 = ~(w0 ^ w3);
+        x1 = ~(w1 ^ w3);
+        x2 = ~(w2 ^ w3);
+    }
+    constexpr uint32_t M = 0x11111111u;
+    uint32_t R[4][2][2];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        // nibble n of S = 3-bit level index of weight 4n + r
+        const uint32_t a = x0 >> r;
+        const uint32_t b = (r >= 1) ? (x1 >> (r >= 1 ? r - 1 : 0)) : (x1 << 1);
+        const uint32_t c = (r >= 2) ? (x2 >> (r >= 2 ? r - 2 : 0)) : (x2 << (r >= 2 ? 0 : 2 - r));
+        const uint32_t S = (a & M) | (b & (M << 1)) | (c & (M << 2));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t sel = h ? (S >> 16) : S;  // weights 16h + 4m + r, m = 0..3
+            uint32_t hb = prmt(t.th0, t.th1, sel);
+            const uint32_t lb = prmt(t.tl0, t.tl1, sel);
+            if (Q4) {
+                // bytes of `flip` = 0xFF where the weight's b_4 is -1: bring the four bits to byte
+                // MSBs (m = 0, 2 in one copy, m = 1, 3 in the other) and replicate them with PRMT
+                const int p0 = 16 * h + r;
+                const uint32_t s02 = (p0 <= 7) ? (nf << (p0 <= 7 ? 7 - p0 : 0)) : (nf >> (p0 > 7 ? p0 - 7 : 0));
+                const uint32_t s13 = (p0 <= 3) ? (nf << (p0 <= 3 ? 3 - p0 : 0)) : (nf >> (p0 > 3 ? p0 - 3 : 0));
+                const uint32_t flip = prmt(s02, s13, 0xD9C8u);
+                hb ^= flip & 0x80808080u;
+            }
+            R[r][h][0] = prmt(lb, hb, 0x5140u);  // weights m = 0, 1
+            R[r][h][1] = prmt(lb, hb, 0x7362u);  // weights m = 2, 3
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            ptx::st_shared_v4(line + (((chunk0 + 2 * h + u) ^ lx) << 4), R[0][h][u], R[1][h][u], R[2][h][u],
+                              R[3][h][u]);
+}
+
+// Same result through fp32 sums, any q <= 8.  w[i] = plane words, a[i] = scales.
+__device__ __forceinline__ void expand32_sum(const uint32_t (&w)[BCQ_MAX_Q], const float (&a)[BCQ_MAX_Q],
+                                             int q, uint32_t line, uint32_t lx, uint32_t chunk0) {
+    float v[32];
+#pragma unroll
+    for (int p = 0; p < 32; ++p) v[p] = 0.0f;
+#pragma unroll
+    for (int i = 0; i < BCQ_MAX_Q; ++i) {
+        if (i < q) {
+            const uint32_t ai = __float_as_uint(a[i]);
+            const uint32_t nw = ~w[i];
+#pragma unroll
+            for (int p = 0; p < 32; ++p) v[p] += __uint_as_float(ai ^ ((nw << (31 - p)) & 0x80000000u));
+        }
+    }
+#pragma unroll
+    for (int cc = 0; cc < 4; ++cc)
+        ptx::st_shared_v4(line + (((chunk0 + cc) ^ lx) << 4), pack_half2(v[8 * cc + 0], v[8 * cc + 4]),
+                          pack_half2(v[8 * cc + 1], v[8 * cc + 5]), pack_half2(v[8 * cc + 2], v[8 * cc + 6]),
+                          pack_half2(v[8 * cc + 3], v[8 * cc + 7]));
+}
+
+template <int QM>
+struct NumWords {
+    static constexpr int value = (QM == QM_GENERIC) ? BCQ_MAX_Q : 4;
+};
+
+// The scales of one (row, group), already multiplied by the weight scale; loaded ahead of use.
+template <int QM>
+struct AlphaSet {
+    float a[NumWords<QM>::value];
+    int key;  // row * G + group, or -1 for a row outside the matrix (expands to zeros)
+};
+
+template <int QM>
+__device__ __forceinline__ void load_alpha(AlphaSet<QM>& s, const float* __restrict__ alpha,
+                                           long long plane_alpha, int G, int q, int j, int c, bool valid,
+                                           float wscale) {
+    s.key = valid ? j * G + c : -1;
+#pragma unroll
+    for (int i = 0; i < NumWords<QM>::value; ++i)
+        s.a[i] = (i < q && valid) ? __ldg(alpha + i * plane_alpha + (long long)j * G + c) * wscale : 0.0f;
+}
+
+// Expands the 32 weights whose plane words sit in shared memory at bits_addr + i * plane_stride.
+template <int QM>
+__device__ __forceinline__ void expand_task(const AlphaSet<QM>& as, uint32_t bits_addr, uint32_t plane_stride,
+                                            Lut& lut, int& lut_key, int q, uint32_t line, uint32_t lx,
+                                            uint32_t chunk0) {
+    uint32_t w[NumWords<QM>::value];
+#pragma unroll
+    for (int i = 0; i < NumWords<QM>::value; ++i)
+        w[i] = (i < q) ? ptx::ld_shared_u32(bits_addr + i * plane_stride) : 0u;
+    if (QM == QM_GENERIC) {
+        uint32_t w8[BCQ_MAX_Q];
+        float a8[BCQ_MAX_Q];
+#pragma unroll
+        for (int i = 0; i < BCQ_MAX_Q; ++i) {
+            w8[i] = w[i % NumWords<QM>::value];
+            a8[i] = as.a[i % NumWords<QM>::value];
+        }
+        expand32_sum(w8, a8, q, line, lx, chunk0);
+    } else {
+        if (as.key != lut_key) {
+            lut = (QM == QM_LUT4) ? build_lut(as.a[0], as.a[1], as.a[2], as.a[3])
+                                  : build_lut(as.a[0], as.a[1], as.a[2], 0.0f);
+            lut_key = as.key;
+        }
+        expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, line, lx, chunk0);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// pre-pass: activations -> fp16 with a per-token power-of-two scale; max |alpha|
+// ------------------------------------------------------------------------------------------
+
+struct WsHeader {
+    uint32_t alpha_max_bits;  // bits of max |alpha| (atomicMax on the unsigned bit pattern)
+    uint32_t pad[3];
+};
+
+struct PrepParams {
+    int n, K, permute, act_blocks;
+    long long ld_in, ld_out;
+    const __nv_bfloat16* in;
+    __half* out;
+    float* tok_inv_scale;  // [n]
+    const float* alpha;
+    long long alpha_count;
+    WsHeader* hdr;
+};
+
+__global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
+    __shared__ uint32_t red[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x >= p.act_blocks) {
+        // ---- max |alpha|
+        const long long nb = gridDim.x - p.act_blocks;
+        uint32_t m = 0u;
+        for (long long i = ((long long)blockIdx.x - p.act_blocks) * 256 + threadIdx.x; i < p.alpha_count;
+             i += nb * 256)
+            m = max(m, __float_as_uint(__ldg(p.alpha + i)) & 0x7FFFFFFFu);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0 && m != 0u) atomicMax(&p.hdr->alpha_max_bits, m);
+        return;
+    }
+    // ---- one token row
+    const int t = blockIdx.x;
+    const uint4* src = reinterpret_cast<const uint4*>(p.in + (long long)t * p.ld_in);
+    uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)t * p.ld_out);
+    const int nvec = (p.K + 7) / 8;
+    uint32_t m = 0u;
+    for (int v = threadIdx.x; v < nvec; v += 256) {
+        const uint4 x = __ldg(src + v);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t b = (xs[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu;
+            if (v * 8 + e < p.K) m = max(m, b);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    m = 0u;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) m = max(m, red[w]);
+    const int sh = shift_for(exponent_of_bits(m << 16), 14);
+    const float scale = pow2f(sh);
+    if (threadIdx.x == 0) p.tok_inv_scale[t] = pow2f(-sh);
+    for (int v = threadIdx.x; v < nvec; v += 256) {
+        const uint4 x = __ldg(src + v);
+        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const uint32_t b = (xs[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu;
+            f[e] = (v * 8 + e < p.K) ? __uint_as_float(b << 16) * scale : 0.0f;
+        }
+        uint4 o;
+        if (p.permute) {
+            o.x = pack_half2(f[0], f[4]);
+            o.y = pack_half2(f[1], f[5]);
+            o.z = pack_half2(f[2], f[6]);
+            o.w = pack_half2(f[3], f[7]);
+        } else {
+            o.x = pack_half2(f[0], f[1]);
+            o.y = pack_half2(f[2], f[3]);
+            o.z = pack_half2(f[4], f[5]);
+            o.w = pack_half2(f[6], f[7]);
+        }
+        dst[v] = o;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// forward / dX for n > 16: A expanded from the bit-planes, B (fp16 activations) by TMA
+// ------------------------------------------------------------------------------------------
+
+struct ExpandParams {
+    int d_out, d_in, q, g, G, pitch, n;
+    int Mdim;          // d_out (fwd) or d_in (dX)
+    int num_kb;        // K blocks of 64 over d_in (fwd) or d_out (dX)
+    int kb_per_split;
+    int splits;
+    const float* alpha;
+    const float* bias;           // fwd only, may be null
+    const WsHeader* hdr;         // max |alpha|
+    const float* tok_inv_scale;  // [n]
+    void* out;                   // [n][ldo]
+    long long ldo;
+    int out_bf16;
+    float* partial;              // [splits][n][Mdim] when splits > 1
+};
+
+// One pipeline stage in shared memory: | A tile 16 KiB | B tile TN x 128 B | plane words |.
+// The plane words arrive by TMA as [plane][row][4 words]: 128 weights of `rows` rows, where rows
+// = 128 weight rows for the forward and decode (the stage uses 64 of the 128 weights) and the 64
+// rows j of the K block for dX (the four words are the tile's 128 k).
+template <int MODE, int TN, int QM>
+struct StageLayout {
+    static constexpr int kBitRows = (MODE == MODE_BWDX) ? 64 : 128;
+    static constexpr uint32_t kBBytes = TN * kBlockK * 2;
+    static constexpr uint32_t kBitsOff = kABytes + kBBytes;
+    static constexpr uint32_t kPlaneBytes = kBitRows * 16;
+    static constexpr uint32_t kBitsBytes = NumWords<QM>::value * kPlaneBytes;
+    static constexpr uint32_t kStageBytes = kBitsOff + kBitsBytes;
+};
+
+template <int MODE, int TN, int STAGES, int QM>
+__global__ void __launch_bounds__(kThreads, 1)
+expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_bits,
+                   const ExpandParams p) {
+    using L = StageLayout<MODE, TN, QM>;
+    constexpr uint32_t kStageBytes = L::kStageBytes;
+    // fp16 x fp16 -> fp32; A is MN-major for dX
+    constexpr uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
+                                ~((1u << 7) | (1u << 10));
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t ctl_base = smem_base + STAGES * kStageBytes;
+    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes;
+
+    Ctl ctl;
+    ctl.full = ctl_base;
+    ctl.aready = ctl_base + 8 * STAGES;
+    ctl.empty = ctl_base + 16 * STAGES;
+    ctl.accum = ctl_base + 24 * STAGES;
+    ctl.spare = ctl.accum + 8;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 16);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 20);
+    ctl.device_flag = &g_timeout_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kBlockM;
+    const int t0 = blockIdx.y * TN;
+    const int kb_begin = blockIdx.z * p.kb_per_split;
+    const int kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+    const int iters = kb_end - kb_begin;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(ctl.full + 8 * s, 1);
+            ptx::mbar_init(ctl.aready + 8 * s, kWorkerWarps);
+            ptx::mbar_init(ctl.empty + 8 * s, 1);
+        }
+        ptx::mbar_init(ctl.accum, 1);
+        ptx::mbar_init(ctl.spare, 1);
+        *ctl.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_b);
+        ptx::prefetch_tmap(&tmap_bits);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), TmemCols<TN>::value);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: activation tile + plane words of the stage
+        if (lane == 0) {
+            bool ok = true;
+            int issued = 0;
+            const uint32_t tx = L::kBBytes + (uint32_t)p.q * L::kPlaneBytes;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                const int kb = kb_begin + it;
+                ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
+                if (!ok) break;
+                const uint32_t st = smem_base + s * kStageBytes;
+                ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, tx);
+                ptx::tma_load_2d(st + kABytes, &tmap_b, kb * kBlockK, t0, ctl.full + 8 * s);
+                if (MODE == MODE_FWD)
+                    ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, (kb >> 1) * 4, m0, 0, ctl.full + 8 * s);
+                else
+                    ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, m0 >> 5, kb * kBlockK, 0, ctl.full + 8 * s);
+                issued = it + 1;
+            }
+            if (!ok)  // giving up: let the copies already issued land before the CTA exits
+                for (int it = max(0, issued - STAGES); it < issued; ++it)
+                    wait_bar(ctl.full + 8 * (it % STAGES), (it / STAGES) & 1, ctl, 2);
+        }
+    } else if (warp == 1) {
+        // ---------------- UMMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 3) && wait_bar(ctl.aready + 8 * s, ph, ctl, 4);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t sa = smem_base + s * kStageBytes;
+                const uint32_t sb = sa + kABytes;
+#pragma unroll
+                for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                    const uint64_t da = (MODE == MODE_FWD) ? ptx::make_smem_desc(sa + kk * 32, 16, 1024)
+                                                           : ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
+                    const uint64_t db = ptx::make_smem_desc(sb + kk * 32, 16, 1024);
+                    ptx::umma_bf16(tmem_base, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::umma_commit(ctl.empty + 8 * s);
+            }
+            if (ok) {
+                ptx::umma_commit(ctl.accum);
+            } else {
+                ptx::umma_commit(ctl.spare);
+                wait_bar(ctl.spare, 0, ctl, 5);
+            }
+        }
+    } else {
+        // ---------------- workers: expansion, then epilogue
+        const int wid = warp - kWorkerWarp0;  // 0..7
+        const long long plane_alpha = (long long)p.d_out * p.G;
+
+        // power of two for the weights: q * max|alpha| lands in [2^13, 2^14)
+        const float amax = __uint_as_float(__ldg(&p.hdr->alpha_max_bits));
+        const int wsh = shift_for(exponent_of_bits(__float_as_uint(amax * (float)p.q)), 13);
+        const float wscale = pow2f(wsh);
+        const float winv = pow2f(-wsh);
+
+        Lut lut = {0u, 0u, 0u, 0u};
+        int lut_key = -2;
+        bool ok = true;
+
+        if (MODE == MODE_FWD) {
+            // task = (weight row, 32-wide half of the stage's 64 k).  The two halves of a row sit
+            // in adjacent lanes, so their scale loads coalesce.  The row's scales change only when
+            // k crosses a group boundary: the set for the next group is loaded when the current
+            // one is taken into use.
+            const int row = wid * 16 + (lane >> 1);
+            const int half = lane & 1;
+            const int j = m0 + row;
+            const bool valid = j < p.d_out;
+            const uint32_t line_off = row * 128, lx = row & 7, chunk0 = half * 4;
+            const int cstep = max(1, kBlockK / p.g);
+            auto group_of = [&](int kb) { return min((kb * kBlockK + half * 32) / p.g, p.G - 1); };
+            AlphaSet<QM> cur, nxt;
+            int c_cur = (iters > 0) ? group_of(kb_begin) : 0;
+            load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
+            load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
+            for (int it = 0; it < iters; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                const int kb = kb_begin + it;
+                const int c = group_of(kb);
+                if (c != c_cur) {
+                    cur = nxt;
+                    c_cur = c;
+                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c + cstep, p.G - 1), valid, wscale);
+                }
+                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // plane words of the stage have landed
+                if (!ok) break;
+                const uint32_t st = smem_base + s * kStageBytes;
+                expand_task<QM>(cur, st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2), L::kPlaneBytes, lut,
+                                lut_key, p.q, st + line_off, lx, chunk0);
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+            }
+        } else {
+            // task = (K index j = 64*kb + jl, 32-wide quarter of the tile's 128 k).  Rows change with
+            // every stage, so the scales are fetched kPrefetch stages ahead.
+            const int jl = wid * 8 + (lane >> 2);
+            const int part = lane & 3;
+            const uint32_t line_off = ((part >> 1) * 8192) + jl * 128, lx = jl & 7, chunk0 = (part & 1) * 4;
+            const int c = min((m0 + part * 32) / p.g, p.G - 1);
+            AlphaSet<QM> ring[kPrefetch];
+            auto fetch = [&](AlphaSet<QM>& slot, int kb) {
+                const int j = kb * kBlockK + jl;
+                load_alpha<QM>(slot, p.alpha, plane_alpha, p.G, p.q, j, c, j < p.d_out, wscale);
+            };
+#pragma unroll
+            for (int d = 0; d < kPrefetch; ++d)
+                if (d < iters) fetch(ring[d], kb_begin + d);
+            for (int it0 = 0; it0 < iters && ok; it0 += kPrefetch) {
+#pragma unroll
+                for (int d = 0; d < kPrefetch; ++d) {
+                    const int it = it0 + d;
+                    if (it < iters && ok) {
+                        const int s = it % STAGES;
+                        const uint32_t ph = (it / STAGES) & 1;
+                        const AlphaSet<QM> cur = ring[d];
+                        if (it + kPrefetch < iters) fetch(ring[d], kb_begin + it + kPrefetch);
+                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);
+                        if (ok) {
+                            const uint32_t st = smem_base + s * kStageBytes;
+                            expand_task<QM>(cur, st + L::kBitsOff + jl * 16 + (part << 2), L::kPlaneBytes, lut, lut_key,
+                                            p.q, st + line_off, lx, chunk0);
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                        }
+                    }
+                }
+            }
+        }
+
+        // epilogue: D[row, col] -> out[t0 + col][m0 + row]; warp w reads TMEM lanes 32*(w%4)..
+        if (ok) ok = wait_bar(ctl.accum, 0, ctl, 7);
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            const int quarter = warp & 3;
+            const int half = wid >> 2;
+            constexpr int HN = TN / 2;
+            constexpr int CH = 16;
+            int m = m0 + quarter * 32 + lane;
+            if (MODE == MODE_BWDX) {
+                // accumulator row r holds k = 8*(r/8) + {0,4,1,5,2,6,3,7}[r % 8]
+                const int ps = m & 7;
+                m = (m & ~7) | ((ps >> 1) + 4 * (ps & 1));
+            }
+            const bool m_ok = m < p.Mdim;
+            const float bias =
+                (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m_ok) ? __ldg(p.bias + m) : 0.0f;
+#pragma unroll 1
+            for (int cb = 0; cb < HN; cb += CH) {
+                const int col = half * HN + cb;
+                if (t0 + col >= p.n) break;  // uniform in the warp
+                uint32_t v[CH];
+                ptx::tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, v);
+                ptx::tmem_ld_wait();
+                if (m_ok) {
+#pragma unroll
+                    for (int cidx = 0; cidx < CH; ++cidx) {
+                        const int t = t0 + col + cidx;
+                        if (t < p.n) {
+                            const float val = __uint_as_float(v[cidx]) * (winv * __ldg(p.tok_inv_scale + t));
+                            if (p.splits > 1) {
+                                p.partial[((long long)blockIdx.z * p.n + t) * p.Mdim + m] = val;
+                            } else if (p.out_bf16) {
+                                reinterpret_cast<__nv_bfloat16*>(p.out)[(long long)t * p.ldo + m] =
+                                    __float2bfloat16_rn(val + bias);
+                            } else {
+                                reinterpret_cast<float*>(p.out)[(long long)t * p.ldo + m] = val + bias;
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TmemCols<TN>::value);
+    }
+}
+
+// out[t][m] = sum_z partial[z][t][m] (+ bias[m]), in the order z = 0, 1, ...
+__global__ void splitk_reduce_kernel(int n, int Mdim, int splits, const float* __restrict__ partial,
+                                     const float* __restrict__ bias, void* out, long long ldo,
+                                     int out_bf16) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long total = (long long)n * Mdim;
+    if (idx >= total) return;
+    const int t = (int)(idx / Mdim);
+    const int m = (int)(idx - (long long)t * Mdim);
+    float s = 0.0f;
+    for (int z = 0; z < splits; ++z) s += __ldg(partial + (long long)z * total + idx);
+    if (bias != nullptr) s += __ldg(bias + m);
+    if (out_bf16)
+        reinterpret_cast<__nv_bfloat16*>(out)[(long long)t * ldo + m] = __float2bfloat16_rn(s);
+    else
+        reinterpret_cast<float*>(out)[(long long)t * ldo + m] = s;
+}
+
+// ------------------------------------------------------------------------------------------
+// decode: n <= 16 tokens, no pre-pass; the workers write both operands
+// ------------------------------------------------------------------------------------------
+
+struct DecodeParams {
+    int d_out, d_in, q, g, G, pitch, n;
+    int num_kb, kb_per_split, splits;
+    const float* alpha;
+    const float* bias;
+    const __nv_bfloat16* X;
+    long long ldx;
+    void* out;
+    long long ldo;
+    int out_bf16;
+    float* partial;  // [splits][n][d_out]
+};
+
+constexpr int kDecTN = 16;
+constexpr int kDecStages = 4;
+
+// Scale of one weight row in decode: the scales of the row's first groups inside the CTA's K slice
+// (at most four) are sampled; their maximum times q is brought to 2^9, which leaves a factor of
+// 64 of headroom for larger scales further along the row before fp16 would overflow.
+__device__ __forceinline__ int decode_row_shift(const float* __restrict__ alpha, long long plane_alpha, int G,
+                                                int q, int j, int c_lo, int c_hi) {
+    uint32_t am = 0u;
+    for (int i = 0; i < q; ++i)
+        for (int c = c_lo; c <= min(c_hi, c_lo + 3); ++c)
+            am = max(am, __float_as_uint(__ldg(alpha + i * plane_alpha + (long long)j * G + c)) & 0x7FFFFFFFu);
+    return shift_for(exponent_of_bits(__float_as_uint(__uint_as_float(am) * (float)q)), 9);
+}
+
+template <int QM>
+__global__ void __launch_bounds__(kThreads, 2)
+decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams p) {
+    using L = StageLayout<MODE_FWD, kDecTN, QM>;
+    constexpr int STAGES = kDecStages;
+    constexpr uint32_t kStageBytes = L::kStageBytes;
+    constexpr uint32_t kIdesc = ptx::make_idesc_bf16(kBlockM, kDecTN, 0, 0) & ~((1u << 7) | (1u << 10));
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t ctl_base = smem_base + STAGES * kStageBytes;
+    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes;
+
+    Ctl ctl;
+    ctl.full = ctl_base;
+    ctl.aready = ctl_base + 8 * STAGES;
+    ctl.empty = ctl_base + 16 * STAGES;
+    ctl.accum = ctl_base + 24 * STAGES;
+    ctl.spare = ctl.accum + 8;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 16);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 20);
+    ctl.device_flag = &g_timeout_flag;
+    float* tok_scale = reinterpret_cast<float*>(ctl_gen + 24 * STAGES + 32);  // [16] scale, [16] inverse
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kBlockM;
+    const int kb_begin = blockIdx.y * p.kb_per_split;
+    const int kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
+    const int iters = kb_end - kb_begin;
+    const int k_lo = kb_begin * kBlockK;
+    const int k_hi = min(kb_end * kBlockK, p.d_in);
+    const int c_lo = min(k_lo / p.g, p.G - 1), c_hi = min((k_hi - 1) / p.g, p.G - 1);
+    const long long plane_alpha = (long long)p.d_out * p.G;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(ctl.full + 8 * s, 1);
+            ptx::mbar_init(ctl.aready + 8 * s, kWorkerWarps);
+            ptx::mbar_init(ctl.empty + 8 * s, 1);
+        }
+        ptx::mbar_init(ctl.accum, 1);
+        ptx::mbar_init(ctl.spare, 1);
+        *ctl.abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_bits);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), TmemCols<kDecTN>::value);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: plane words only
+        if (lane == 0) {
+            bool ok = true;
+            int issued = 0;
+            const uint32_t tx = (uint32_t)p.q * L::kPlaneBytes;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                const int kb = kb_begin + it;
+                ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 20);
+                if (!ok) break;
+                ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, tx);
+                ptx::tma_load_3d(smem_base + s * kStageBytes + L::kBitsOff, &tmap_bits, (kb >> 1) * 4, m0, 0,
+                                 ctl.full + 8 * s);
+                issued = it + 1;
+            }
+            if (!ok)
+                for (int it = max(0, issued - STAGES); it < issued; ++it)
+                    wait_bar(ctl.full + 8 * (it % STAGES), (it / STAGES) & 1, ctl, 25);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1;
+                ok = wait_bar(ctl.aready + 8 * s, ph, ctl, 21);
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t sa = smem_base + s * kStageBytes;
+                const uint32_t sb = sa + kABytes;
+#pragma unroll
+                for (int kk = 0; kk < kBlockK / 16; ++kk)
+                    ptx::umma_bf16(tmem_base, ptx::make_smem_desc(sa + kk * 32, 16, 1024),
+                                   ptx::make_smem_desc(sb + kk * 32, 16, 1024), kIdesc,
+                                   (it > 0 || kk > 0) ? 1u : 0u);
+                ptx::umma_commit(ctl.empty + 8 * s);
+            }
+            if (ok) {
+                ptx::umma_commit(ctl.accum);
+            } else {
+                ptx::umma_commit(ctl.spare);
+                wait_bar(ctl.spare, 0, ctl, 22);
+            }
+        }
+    } else {
+        const int wid = warp - kWorkerWarp0;
+        const int e = wid * 32 + lane;  // 0..255
+        const int row = wid * 16 + (lane >> 1);
+        const int half = lane & 1;
+        const int j = m0 + row;
+        const bool valid = j < p.d_out;
+        const uint32_t lx = row & 7;
+
+        // ---- per-token scale over this CTA's K slice: thread = (token e / 16, every 16th vector)
+        {
+            const int t = e >> 4, sub = e & 15;
+            uint32_t m = 0u;
+            if (t < p.n) {
+                const __nv_bfloat16* xrow = p.X + (long long)t * p.ldx;
+                for (int k = k_lo + sub * 8; k < k_hi; k += 128) {
+                    const uint4 x = __ldg(reinterpret_cast<const uint4*>(xrow + k));
+                    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                    for (int el = 0; el < 8; ++el)
+                        if (k + el < p.d_in) m = max(m, (xs[el >> 1] >> ((el & 1) * 16)) & 0x7FFFu);
+                }
+            }
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (sub == 0) {
+                const int sh = shift_for(exponent_of_bits(m << 16), 14);
+                tok_scale[t] = pow2f(sh);
+                tok_scale[16 + t] = pow2f(-sh);
+            }
+        }
+        const float wscale = valid ? pow2f(decode_row_shift(p.alpha, plane_alpha, p.G, p.q, j, c_lo, c_hi)) : 1.0f;
+        asm volatile("bar.sync 1, %0;" ::"n"(kWorkers) : "memory");  // tok_scale visible to all workers
+
+        // activation task of threads e < 128: (token e / 8, 8 consecutive k = one 16-byte chunk)
+        const int xt = e >> 3, xch = e & 7;
+        const bool x_task = e < 128;
+        const float xscale = x_task ? tok_scale[xt] : 0.0f;
+        auto fetch_x = [&](uint4& slot, int kb) {
+            const int k = kb * kBlockK + xch * 8;
+            slot = make_uint4(0u, 0u, 0u, 0u);
+            if (x_task && xt < p.n && k < p.d_in)
+                slot = __ldg(reinterpret_cast<const uint4*>(p.X + (long long)xt * p.ldx + k));
+        };
+
+        const int cstep = max(1, kBlockK / p.g);
+        auto group_of = [&](int kb) { return min((kb * kBlockK + half * 32) / p.g, p.G - 1); };
+        AlphaSet<QM> cur, nxt;
+        int c_cur = (iters > 0) ? group_of(kb_begin) : 0;
+        load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
+        load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
+        uint4 xring[kPrefetch];
+#pragma unroll
+        for (int d = 0; d < kPrefetch; ++d)
+            if (d < iters) fetch_x(xring[d], kb_begin + d);
+
+        Lut lut = {0u, 0u, 0u, 0u};
+        int lut_key = -2;
+        bool ok = true;
+        for (int it0 = 0; it0 < iters && ok; it0 += kPrefetch) {
+#pragma unroll
+            for (int d = 0; d < kPrefetch; ++d) {
+                const int it = it0 + d;
+                if (it < iters && ok) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1;
+                    const int kb = kb_begin + it;
+                    const uint4 xcur = xring[d];
+                    if (it + kPrefetch < iters) fetch_x(xring[d], kb + kPrefetch);
+                    const int c = group_of(kb);
+                    if (c != c_cur) {
+                        cur = nxt;
+                        c_cur = c;
+                        load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c + cstep, p.G - 1), valid, wscale);
+                    }
+                    ok = wait_bar(ctl.full + 8 * s, ph, ctl, 23);
+                    if (ok) {
+                        const uint32_t st = smem_base + s * kStageBytes;
+                        expand_task<QM>(cur, st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2), L::kPlaneBytes,
+                                        lut, lut_key, p.q, st + row * 128, lx, half * 4);
+                        if (x_task) {
+                            const uint32_t xs[4] = {xcur.x, xcur.y, xcur.z, xcur.w};
+                            float f[8];
+#pragma unroll
+                            for (int el = 0; el < 8; ++el) {
+                                const uint32_t b = (xs[el >> 1] >> ((el & 1) * 16)) & 0xFFFFu;
+                                f[el] = (kb * kBlockK + xch * 8 + el < p.d_in) ? __uint_as_float(b << 16) * xscale
+                                                                             : 0.0f;
+                            }
+                            ptx::st_shared_v4(st + kABytes + xt * 128 + ((xch ^ (xt & 7)) << 4),
+                                              pack_half2(f[0], f[4]), pack_half2(f[1], f[5]),
+                                              pack_half2(f[2], f[6]), pack_half2(f[3], f[7]));
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                    }
+                }
+            }
+        }
+
+        // ---- epilogue: thread = (TMEM lane = weight row, tokens 8*eh .. 8*eh+7)
+        if (ok) ok = wait_bar(ctl.accum, 0, ctl, 24);
+        const int quarter = warp & 3, eh = wid >> 2;
+        if (ok && eh * 8 < p.n) {
+            ptx::tc_fence_after_sync();
+            uint32_t v[8];
+            ptx::tmem_ld_x8(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(eh * 8), v);
+            ptx::tmem_ld_wait();
+            const int je = m0 + quarter * 32 + lane;
+            if (je < p.d_out) {
+                const float winv = pow2f(-decode_row_shift(p.alpha, plane_alpha, p.G, p.q, je, c_lo, c_hi));
+                const float bias = (p.bias != nullptr && p.splits == 1) ? __ldg(p.bias + je) : 0.0f;
+#pragma unroll
+                for (int cidx = 0; cidx < 8; ++cidx) {
+                    const int t = eh * 8 + cidx;
+                    if (t < p.n) {
+                        const float val = __uint_as_float(v[cidx]) * (winv * tok_scale[16 + t]);
+                        if (p.splits > 1)
+                            p.partial[((long long)blockIdx.y * p.n + t) * p.d_out + je] = val;
+                        else if (p.out_bf16)
+                            reinterpret_cast<__nv_bfloat16*>(p.out)[(long long)t * p.ldo + je] =
+                                __float2bfloat16_rn(val + bias);
+                        else
+                            reinterpret_cast<float*>(p.out)[(long long)t * p.ldo + je] = val + bias;
+                    }
+                }
+            }
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, TmemCols<kDecTN>::value);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------
+
+struct ExpandPlan {
+    int TN, splits, kb_per_split, num_kb, m_tiles, n_tiles;
+    size_t off_tok, off_act, off_partial, total;  // workspace layout (bytes)
+    int ld_act;                                   // pitch of the fp16 activations (elements)
+};
+
+// Tile width over tokens and the K split.  Wide token tiles amortise the expansion of a weight
+// tile over more tokens; the K split fills the SMs when the output has few tiles.
+ExpandPlan plan_expand(int Mdim, int Kdim, int n) {
+    ExpandPlan pl;
+    const int sms = sm_count();
+    pl.m_tiles = ceil_div(Mdim, kBlockM);
+    pl.num_kb = ceil_div(Kdim, kBlockK);
+    int tn;
+    if (n <= 32) tn = 32;
+    else if (n <= 64) tn = 64;
+    else if (n <= 128) tn = 128;
+    else {
+        tn = 256;
+        if (pl.m_tiles * ceil_div(n, 256) < sms) tn = 128;
+    }
+    pl.TN = tn;
+    pl.n_tiles = ceil_div(n, tn);
+    const int tiles = pl.m_tiles * pl.n_tiles;
+    int splits = sms / tiles;
+    if (splits < 1) splits = 1;
+    const int max_splits = (pl.num_kb + 3) / 4;  // at least 4 K blocks per CTA
+    if (splits > max_splits) splits = max_splits;
+    if (splits > 32) splits = 32;
+    pl.kb_per_split = ceil_div(pl.num_kb, splits);
+    pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
+    pl.ld_act = (int)align_up((size_t)Kdim, 8);
+    pl.off_tok = sizeof(WsHeader);
+    pl.off_act = align_up(pl.off_tok + (size_t)n * sizeof(float), 128);
+    pl.off_partial = align_up(pl.off_act + (size_t)n * pl.ld_act * 2, 128);
+    pl.total = pl.off_partial + (pl.splits > 1 ? (size_t)pl.splits * n * Mdim * sizeof(float) : 0);
+    return pl;
+}
+
+struct DecodePlan {
+    int m_tiles, num_kb, splits, kb_per_split;
+    size_t total;
+};
+
+DecodePlan plan_decode(int d_out, int d_in, int n) {
+    DecodePlan pl;
+    const int sms = sm_count();
+    pl.m_tiles = ceil_div(d_out, kBlockM);
+    pl.num_kb = ceil_div(d_in, kBlockK);
+    int splits = (2 * sms) / pl.m_tiles;  // 72 KiB of shared memory per CTA: several CTAs per SM
+    if (splits < 1) splits = 1;
+    const int max_splits = (pl.num_kb + 7) / 8;  // at least 8 K blocks per CTA
+    if (splits > max_splits) splits = max_splits;
+    if (splits > 64) splits = 64;
+    pl.kb_per_split = ceil_div(pl.num_kb, splits);
+    pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
+    pl.total = pl.splits > 1 ? (size_t)pl.splits * n * d_out * sizeof(float) : 0;
+    return pl;
+}
+
+constexpr size_t kSmemBudget = 232448 - 1024 - 512;  // 227 KiB minus alignment slack and the control block
+
+template <int MODE, int TN, int QM>
+constexpr int stages_for() {
+    constexpr size_t per = StageLayout<MODE, TN, QM>::kStageBytes;
+    constexpr int fit = (int)(kSmemBudget / per);
+    return fit > 6 ? 6 : fit;
+}
+
+template <int MODE, int TN, int QM>
+constexpr size_t smem_for() {
+    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + 512;
+}
+
+template <int MODE, int TN, int QM>
+bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tm_bits, const ExpandParams& p,
+                         const ExpandPlan& pl, cudaStream_t stream) {
+    auto kern = expand_gemm_kernel<MODE, TN, stages_for<MODE, TN, QM>(), QM>;
+    constexpr size_t smem = smem_for<MODE, TN, QM>();
+    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.n_tiles, (unsigned)pl.splits);
+    kern<<<grid, kThreads, smem, stream>>>(tm, tm_bits, p);
+    BCQ_CUDA_TRY(cudaGetLastError());
+    return BCQ_OK;
+}
+
+template <int MODE, int TN>
+bcq_status launch_expand_q(const CUtensorMap& tm, const CUtensorMap& tm_bits, const ExpandParams& p,
+                           const ExpandPlan& pl, cudaStream_t stream) {
+    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, tm_bits, p, pl, stream);
+    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, tm_bits, p, pl, stream);
+    return launch_expand<MODE, TN, QM_GENERIC>(tm, tm_bits, p, pl, stream);
+}
+
+// act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).
+template <int MODE>
+bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act, size_t ldact,
+                      const uint32_t* bits, const float* alpha, const float* bias, void* out, size_t ldo,
+                      int out_dtype, void* ws, size_t ws_bytes, void* stream) {
+    const int Mdim = (MODE == MODE_FWD) ? d_out : d_in;
+    const int Kdim = (MODE == MODE_FWD) ? d_in : d_out;
+    const ExpandPlan pl = plan_expand(Mdim, Kdim, n);
+    if (ws == nullptr) return BCQ_ERR_NULL;
+    if (ws_bytes < pl.total) return BCQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return BCQ_ERR_ALIGN;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint8_t* wsb = reinterpret_cast<uint8_t*>(ws);
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(wsb);
+    float* tok = reinterpret_cast<float*>(wsb + pl.off_tok);
+    __half* act16 = reinterpret_cast<__half*>(wsb + pl.off_act);
+    const int pitch = (int)bcq_pitch_words(d_in);
+
+    CUtensorMap tm, tm_bits;
+    bcq_status st = make_tmap_16bit(&tm, act16, 1, pl.ld_act, n, (size_t)pl.ld_act, pl.TN);
+    if (st != BCQ_OK) return st;
+    st = make_tmap_bits(&tm_bits, bits, d_out, pitch, q, MODE == MODE_FWD ? 128 : 64);
+    if (st != BCQ_OK) return st;
+
+    BCQ_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s));
+    PrepParams pp;
+    pp.n = n; pp.K = Kdim; pp.permute = (MODE == MODE_FWD) ? 1 : 0; pp.act_blocks = n;
+    pp.ld_in = (long long)ldact; pp.ld_out = pl.ld_act;
+    pp.in = reinterpret_cast<const __nv_bfloat16*>(act); pp.out = act16; pp.tok_inv_scale = tok;
+    pp.alpha = alpha; pp.alpha_count = (long long)bcq_alpha_count(d_out, d_in, q, g); pp.hdr = hdr;
+    long long ablocks = (pp.alpha_count + 256 * 16 - 1) / (256 * 16);
+    if (ablocks > 128) ablocks = 128;
+    if (ablocks < 1) ablocks = 1;
+    prepare_kernel<<<(unsigned)(n + ablocks), 256, 0, s>>>(pp);
+    BCQ_CUDA_TRY(cudaGetLastError());
+
+    ExpandParams p;
+    p.d_out = d_out; p.d_in = d_in; p.q = q; p.g = g;
+    p.G = (int)bcq_num_groups(d_in, g);
+    p.pitch = pitch;
+    p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
+    p.alpha = alpha; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
+    p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
+    p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
+    switch (pl.TN) {
+        case 32: st = launch_expand_q<MODE, 32>(tm, tm_bits, p, pl, s); break;
+        case 64: st = launch_expand_q<MODE, 64>(tm, tm_bits, p, pl, s); break;
+        case 128: st = launch_expand_q<MODE, 128>(tm, tm_bits, p, pl, s); break;
+        default: st = launch_expand_q<MODE, 256>(tm, tm_bits, p, pl, s); break;
+    }
+    if (st != BCQ_OK) return st;
+    if (pl.splits > 1) {
+        const long long total = (long long)n * Mdim;
+        splitk_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+            n, Mdim, pl.splits, p.partial, bias, out, (long long)ldo, p.out_bf16);
+        BCQ_CUDA_TRY(cudaGetLastError());
+    }
+    return BCQ_OK;
+}
+
+template <int QM>
+bcq_status launch_decode(const CUtensorMap& tm_bits, const DecodeParams& p, const DecodePlan& pl,
+                         cudaStream_t s) {
+    constexpr size_t smem = (size_t)kDecStages * StageLayout<MODE_FWD, kDecTN, QM>::kStageBytes + 1024 + 512;
+    auto kern = decode_kernel<QM>;
+    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.splits);
+    kern<<<grid, kThreads, smem, s>>>(tm_bits, p);
+    BCQ_CUDA_TRY(cudaGetLastError());
+    return BCQ_OK;
+}
+
+bcq_status run_decode(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                      const uint32_t* bits, const float* alpha, const float* bias, void* Y, size_t ldy,
+                      int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+    const DecodePlan pl = plan_decode(d_out, d_in, n);
+    if (pl.total > 0) {
+        if (ws == nullptr) return BCQ_ERR_NULL;
+        if (ws_bytes < pl.total) return BCQ_ERR_WORKSPACE;
+        if (!aligned16(ws)) return BCQ_ERR_ALIGN;
+    }
+    DecodeParams p;
+    p.d_out = d_out; p.d_in = d_in; p.q = q; p.g = g;
+    p.G = (int)bcq_num_groups(d_in, g);
+    p.pitch = (int)bcq_pitch_words(d_in);
+    p.n = n; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
+    p.alpha = alpha; p.bias = bias;
+    p.X = reinterpret_cast<const __nv_bfloat16*>(X); p.ldx = (long long)ldx;
+    p.out = Y; p.ldo = (long long)ldy; p.out_bf16 = (y_dtype == BCQ_BF16);
+    p.partial = reinterpret_cast<float*>(ws);
+    CUtensorMap tm_bits;
+    bcq_status st = make_tmap_bits(&tm_bits, bits, d_out, p.pitch, q, 128);
+    if (st != BCQ_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (q <= 3) st = launch_decode<QM_LUT3>(tm_bits, p, pl, s);
+    else if (q == 4) st = launch_decode<QM_LUT4>(tm_bits, p, pl, s);
+    else st = launch_decode<QM_GENERIC>(tm_bits, p, pl, s);
+    if (st != BCQ_OK) return st;
+    if (pl.splits > 1) {
+        const long long total = (long long)n * d_out;
+        splitk_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+            n, d_out, pl.splits, p.partial, bias, Y, (long long)ldy, p.out_bf16);
+        BCQ_CUDA_TRY(cudaGetLastError());
+    }
+    return BCQ_OK;
+}
+
+bcq_status fwd_common(int decode, int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                      const uint32_t* bits, const float* alpha, const float* bias, void* Y, size_t ldy,
+                      int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+    bcq_status st = check_shape(d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1 || (decode && n > 16)) return BCQ_ERR_SHAPE;
+    if (!bits || !alpha || !Y) return BCQ_ERR_NULL;
+    if ((st = check_act(X, ldx, d_in)) != BCQ_OK) return st;
+    if (ldy < (size_t)d_out) return BCQ_ERR_SHAPE;
+    if (y_dtype != BCQ_F32 && y_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
+    if (!aligned16(bits)) return BCQ_ERR_ALIGN;
+    if (decode)
+        return run_decode(d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes, stream);
+    return run_expand<MODE_FWD>(d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes,
+                                stream);
+}
+
+}  // namespace
+
+namespace bcq {
+bcq_status expand_timeout_flag(int* flag_out, int reset) {
+    int v = 0;
+    BCQ_CUDA_TRY(cudaMemcpyFromSymbol(&v, g_timeout_flag, sizeof(int)));
+    *flag_out = v;
+    if (reset && v != 0) {
+        const int zero = 0;
+        BCQ_CUDA_TRY(cudaMemcpyToSymbol(g_timeout_flag, &zero, sizeof(int)));
+    }
+    return BCQ_OK;
+}
+
+size_t fwd_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_expand(d_out, d_in, n).total; }
+size_t decode_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_decode(d_out, d_in, n).total; }
+size_t bwd_x_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_expand(d_in, d_out, n).total; }
+}  // namespace bcq
+
+extern "C" bcq_status bcq_linear_fwd(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                                     const uint32_t* bits, const float* alpha, const float* bias, void* Y,
+                                     size_t ldy, int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+    return fwd_common(0, d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes,
+                      stream);
+}
+
+extern "C" bcq_status bcq_linear_decode(int d_out, int d_in, int q, int g, int n, const void* X,
+                                        size_t ldx, const uint32_t* bits, const float* alpha,
+                                        const float* bias, void* Y, size_t ldy, int y_dtype, void* ws,
+                                        size_t ws_bytes, void* stream) {
+    return fwd_common(1, d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes,
+                      stream);
+}
+
+extern "C" bcq_status bcq_linear_bwd_x(int d_out, int d_in, int q, int g, int n, const void* dY,
+                                       size_t lddy, const uint32_t* bits, const float* alpha, void* dX,
+                                       size_t lddx, int dx_dtype, void* ws, size_t ws_bytes,
+                                       void* stream) {
+    bcq_status st = check_shape(d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1) return BCQ_ERR_SHAPE;
+    if (!bits || !alpha || !dX) return BCQ_ERR_NULL;
+    if ((st = check_act(dY, lddy, d_out)) != BCQ_OK) return st;
+    if (lddx < (size_t)d_in) return BCQ_ERR_SHAPE;
+    if (dx_dtype != BCQ_F32 && dx_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
+    if (!aligned16(bits)) return BCQ_ERR_ALIGN;
+    return run_expand<MODE_BWDX>(d_out, d_in, q, g, n, dY, lddy, bits, alpha, nullptr, dX, lddx, dx_dtype, ws,
+                                 ws_bytes, stream);
+}

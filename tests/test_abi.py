@@ -71,7 +71,7 @@ def test_argument_validation_happens_before_any_launch():
 
 
 def test_workspace_sizes_are_consistent():
-    # decode splits K over CTAs, so it needs room for the partial sums; big prefill does not
+    # decode splits K over CTAs and needs room for partial sums; prefill holds its fp16 activations
     assert bcq.workspace_bytes(bcq.OP_DECODE, 4096, 16384, 4, 128, 16) > 0
-    assert bcq.workspace_bytes(bcq.OP_FWD, 3072, 1024, 3, 1024, 2048) == 0
+    assert bcq.workspace_bytes(bcq.OP_FWD, 3072, 1024, 3, 1024, 2048) >= 2048 * 1024 * 2
     assert bcq.workspace_bytes(bcq.OP_BWD_ALPHA, 1024, 1024, 3, 1024, 512) > 0
