@@ -153,6 +153,10 @@ bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, int n, const 
 const char* bcq_status_string(int status);
 /* cudaError_t value of the last CUDA failure seen by this library on the calling thread. */
 int bcq_last_cuda_error(void);
+/* Number of GPU kernels this library has launched from the calling thread since it was loaded
+ * (a monotonic counter; memsets are not counted).  Lets a caller state how many of this
+ * library's kernels ran inside a region it timed. */
+unsigned long long bcq_kernel_launches(void);
 /* Reads (and with reset != 0 clears) the device-side flag that kernels set when a bounded wait
  * expired.  Synchronises the device.  *flag_out = 0 means no kernel has given up. */
 bcq_status bcq_device_timeout_flag(int* flag_out /* host */, int reset);

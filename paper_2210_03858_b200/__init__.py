@@ -23,7 +23,8 @@ OP_QUANTIZE, OP_FWD, OP_DECODE, OP_BWD_X, OP_BWD_ALPHA = 0, 1, 2, 3, 4
 SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_count",
            "bcq_payload_bits", "bcq_workspace_bytes", "bcq_quantize", "bcq_dequantize",
            "bcq_linear_fwd", "bcq_linear_decode", "bcq_linear_bwd_x", "bcq_linear_bwd_alpha",
-           "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag")
+           "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag",
+           "bcq_kernel_launches")
 
 
 class BcqError(RuntimeError):
@@ -73,6 +74,8 @@ def lib() -> C.CDLL:
         l.bcq_status_string.argtypes = [i]
         l.bcq_last_cuda_error.restype = i
         l.bcq_last_cuda_error.argtypes = []
+        l.bcq_kernel_launches.restype = C.c_ulonglong
+        l.bcq_kernel_launches.argtypes = []
         l.bcq_device_timeout_flag.restype = i
         l.bcq_device_timeout_flag.argtypes = [C.POINTER(C.c_int), i]
         _lib = l
@@ -230,6 +233,10 @@ def linear_bwd_alpha(dY, X, bits, d_in: int, g: int, plane_mask=None, scale: flo
                                       1 if accumulate else 0, _ptr(out), _ptr(ws), ws_bytes,
                                       _stream()), "bcq_linear_bwd_alpha")
     return out
+
+
+def kernel_launches() -> int:
+    return int(lib().bcq_kernel_launches())
 
 
 def device_timeout_flag(reset: bool = False) -> int:

@@ -3,7 +3,9 @@
 
 namespace bcq {
 static thread_local int t_last_cuda_error = 0;
+static thread_local unsigned long long t_launches = 0;
 void set_last_cuda_error(int e) { t_last_cuda_error = e; }
+void count_launch() { ++t_launches; }
 }  // namespace bcq
 
 extern "C" size_t bcq_pitch_words(int d_in) {
@@ -42,6 +44,8 @@ extern "C" const char* bcq_status_string(int status) {
         default: return "unknown status";
     }
 }
+
+extern "C" unsigned long long bcq_kernel_launches(void) { return bcq::t_launches; }
 
 extern "C" int bcq_last_cuda_error(void) { return bcq::t_last_cuda_error; }
 

@@ -14,6 +14,9 @@ namespace bcq {
 // cudaError_t of the last failing CUDA call on this thread (read by bcq_last_cuda_error()).
 void set_last_cuda_error(int e);
 
+// Called once per kernel launch (bcq_kernel_launches()).
+void count_launch();
+
 inline bcq_status cuda_fail(cudaError_t e) {
     set_last_cuda_error((int)e);
     return BCQ_ERR_CUDA;

@@ -345,17 +345,20 @@ extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, in
         BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)smem_for<256>()));
         kern<<<grid, kThreads, smem_for<256>(), s>>>(tm_dy, tm_x, p);
+    bcq::count_launch();
     } else {
         auto kern = dalpha_kernel<128, stages_for<128>()>;
         BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)smem_for<128>()));
         kern<<<grid, kThreads, smem_for<128>(), s>>>(tm_dy, tm_x, p);
+    bcq::count_launch();
     }
     BCQ_CUDA_TRY(cudaGetLastError());
     const long long total = (long long)q * p.G * d_out;
     dalpha_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
         d_out, d_in, q, g, p.G, pl.HN, pl.splits, pl.n_subtiles, pl.slots, plane_mask, scale, accumulate,
         p.partial, dalpha);
+    bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
 }

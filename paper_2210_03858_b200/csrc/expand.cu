@@ -92,11 +92,11 @@ __device__ __forceinline__ Lut build_lut(float a0, float a1, float a2, float bas
     return t;
 }
 
-// 32 weights of one row from the plane words w0..w3 through the lookup table, stored as four
-// 16-byte chunks (slots chunk0..chunk0+3) of the 128-byte line at `line` (swizzle key lx).
-// Chunk cc holds weights 8cc..8cc+7 in the order 0,4,1,5,2,6,3,7.
+// 16 weights of one row (bits 0..15 of the plane words w0..w3) through the lookup table, stored
+// as two 16-byte chunks (slots chunk0, chunk0 + 1) of the 128-byte line at `line` (swizzle key
+// lx).  Chunk u holds weights 8u..8u+7 in the order 0,4,1,5,2,6,3,7.
 template <bool Q4>
-__device__ __forceinline__ void expand32_lut(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+__device__ __forceinline__ void expand16_lut(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
                                              const Lut& t, uint32_t line, uint32_t lx, uint32_t chunk0) {
     uint32_t x0 = w0, x1 = w1, x2 = w2, nf = 0u;
     if (Q4) {
@@ -107,57 +107,49 @@ __device__ __forceinline__ void expand32_lut(uint32_t w0, uint32_t w1, uint32_t 
         x2 = ~(w2 ^ w3);
     }
     constexpr uint32_t M = 0x11111111u;
-    uint32_t R[4][2][2];
+    uint32_t R[4][2];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         // nibble n of S = 3-bit level index of weight 4n + r
         const uint32_t a = x0 >> r;
         const uint32_t b = (r >= 1) ? (x1 >> (r >= 1 ? r - 1 : 0)) : (x1 << 1);
         const uint32_t c = (r >= 2) ? (x2 >> (r >= 2 ? r - 2 : 0)) : (x2 << (r >= 2 ? 0 : 2 - r));
-        const uint32_t S = (a & M) | (b & (M << 1)) | (c & (M << 2));
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t sel = h ? (S >> 16) : S;  // weights 16h + 4m + r, m = 0..3
-            uint32_t hb = prmt(t.th0, t.th1, sel);
-            const uint32_t lb = prmt(t.tl0, t.tl1, sel);
-            if (Q4) {
-                // bytes of `flip` = 0xFF where the weight's b_4 is -1: bring the four bits to byte
-                // MSBs (m = 0, 2 in one copy, m = 1, 3 in the other) and replicate them with PRMT
-                const int p0 = 16 * h + r;
-                const uint32_t s02 = (p0 <= 7) ? (nf << (p0 <= 7 ? 7 - p0 : 0)) : (nf >> (p0 > 7 ? p0 - 7 : 0));
-                const uint32_t s13 = (p0 <= 3) ? (nf << (p0 <= 3 ? 3 - p0 : 0)) : (nf >> (p0 > 3 ? p0 - 3 : 0));
-                const uint32_t flip = prmt(s02, s13, 0xD9C8u);
-                hb ^= flip & 0x80808080u;
-            }
-            R[r][h][0] = prmt(lb, hb, 0x5140u);  // weights m = 0, 1
-            R[r][h][1] = prmt(lb, hb, 0x7362u);  // weights m = 2, 3
+        const uint32_t S = (a & M) | (b & (M << 1)) | (c & (M << 2));  // PRMT reads the low 16 bits
+        uint32_t hb = prmt(t.th0, t.th1, S);
+        const uint32_t lb = prmt(t.tl0, t.tl1, S);
+        if (Q4) {
+            // bytes of `flip` = 0xFF where the weight's b_4 is -1: bring the four bits (weights r,
+            // r+4, r+8, r+12) to byte MSBs, two per copy, and replicate them with PRMT
+            const uint32_t s02 = nf << (7 - r);
+            const uint32_t s13 = nf << (3 - r);
+            const uint32_t flip = prmt(s02, s13, 0xD9C8u);
+            hb ^= flip & 0x80808080u;
         }
+        R[r][0] = prmt(lb, hb, 0x5140u);  // weights r, r + 4
+        R[r][1] = prmt(lb, hb, 0x7362u);  // weights r + 8, r + 12
     }
 #pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-            ptx::st_shared_v4(line + (((chunk0 + 2 * h + u) ^ lx) << 4), R[0][h][u], R[1][h][u], R[2][h][u],
-                              R[3][h][u]);
+    for (int u = 0; u < 2; ++u)
+        ptx::st_shared_v4(line + (((chunk0 + u) ^ lx) << 4), R[0][u], R[1][u], R[2][u], R[3][u]);
 }
 
-// Same result through fp32 sums, any q <= 8.  w[i] = plane words, a[i] = scales.
-__device__ __forceinline__ void expand32_sum(const uint32_t (&w)[BCQ_MAX_Q], const float (&a)[BCQ_MAX_Q],
+// Same result through fp32 sums, any q <= 8.  w[i] = plane words (bits 0..15 used), a[i] = scales.
+__device__ __forceinline__ void expand16_sum(const uint32_t (&w)[BCQ_MAX_Q], const float (&a)[BCQ_MAX_Q],
                                              int q, uint32_t line, uint32_t lx, uint32_t chunk0) {
-    float v[32];
+    float v[16];
 #pragma unroll
-    for (int p = 0; p < 32; ++p) v[p] = 0.0f;
+    for (int p = 0; p < 16; ++p) v[p] = 0.0f;
 #pragma unroll
     for (int i = 0; i < BCQ_MAX_Q; ++i) {
         if (i < q) {
             const uint32_t ai = __float_as_uint(a[i]);
             const uint32_t nw = ~w[i];
 #pragma unroll
-            for (int p = 0; p < 32; ++p) v[p] += __uint_as_float(ai ^ ((nw << (31 - p)) & 0x80000000u));
+            for (int p = 0; p < 16; ++p) v[p] += __uint_as_float(ai ^ ((nw << (31 - p)) & 0x80000000u));
         }
     }
 #pragma unroll
-    for (int cc = 0; cc < 4; ++cc)
+    for (int cc = 0; cc < 2; ++cc)
         ptx::st_shared_v4(line + (((chunk0 + cc) ^ lx) << 4), pack_half2(v[8 * cc + 0], v[8 * cc + 4]),
                           pack_half2(v[8 * cc + 1], v[8 * cc + 5]), pack_half2(v[8 * cc + 2], v[8 * cc + 6]),
                           pack_half2(v[8 * cc + 3], v[8 * cc + 7]));
@@ -185,15 +177,16 @@ __device__ __forceinline__ void load_alpha(AlphaSet<QM>& s, const float* __restr
         s.a[i] = (i < q && valid) ? __ldg(alpha + i * plane_alpha + (long long)j * G + c) * wscale : 0.0f;
 }
 
-// Expands the 32 weights whose plane words sit in shared memory at bits_addr + i * plane_stride.
+// Expands the 16 weights that start at bit `bit_shift` (0 or 16) of the plane words in shared
+// memory at bits_addr + i * plane_stride.
 template <int QM>
 __device__ __forceinline__ void expand_task(const AlphaSet<QM>& as, uint32_t bits_addr, uint32_t plane_stride,
-                                            Lut& lut, int& lut_key, int q, uint32_t line, uint32_t lx,
-                                            uint32_t chunk0) {
+                                            uint32_t bit_shift, Lut& lut, int& lut_key, int q, uint32_t line,
+                                            uint32_t lx, uint32_t chunk0) {
     uint32_t w[NumWords<QM>::value];
 #pragma unroll
     for (int i = 0; i < NumWords<QM>::value; ++i)
-        w[i] = (i < q) ? ptx::ld_shared_u32(bits_addr + i * plane_stride) : 0u;
+        w[i] = (i < q) ? (ptx::ld_shared_u32(bits_addr + i * plane_stride) >> bit_shift) : 0u;
     if (QM == QM_GENERIC) {
         uint32_t w8[BCQ_MAX_Q];
         float a8[BCQ_MAX_Q];
@@ -202,14 +195,14 @@ __device__ __forceinline__ void expand_task(const AlphaSet<QM>& as, uint32_t bit
             w8[i] = w[i % NumWords<QM>::value];
             a8[i] = as.a[i % NumWords<QM>::value];
         }
-        expand32_sum(w8, a8, q, line, lx, chunk0);
+        expand16_sum(w8, a8, q, line, lx, chunk0);
     } else {
         if (as.key != lut_key) {
             lut = (QM == QM_LUT4) ? build_lut(as.a[0], as.a[1], as.a[2], as.a[3])
                                   : build_lut(as.a[0], as.a[1], as.a[2], 0.0f);
             lut_key = as.key;
         }
-        expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, line, lx, chunk0);
+        expand16_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, line, lx, chunk0);
     }
 }
 
@@ -332,8 +325,14 @@ struct StageLayout {
     static constexpr uint32_t kStageBytes = kBitsOff + kBitsBytes;
 };
 
+// Prefill kernels run 16 worker warps (plus the TMA and UMMA warps): a task is 16 weights of one
+// row, so that four warps per scheduler hide each other's dependency stalls.
+constexpr int kPfWorkerWarps = 16;
+constexpr int kPfWorkers = kPfWorkerWarps * 32;
+constexpr int kPfThreads = (kWorkerWarp0 + kPfWorkerWarps) * 32;
+
 template <int MODE, int TN, int STAGES, int QM>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 1)
 expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_bits,
                    const ExpandParams p) {
     using L = StageLayout<MODE, TN, QM>;
@@ -357,6 +356,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 16);
     ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 20);
     ctl.device_flag = &g_timeout_flag;
+    float* out_scale = reinterpret_cast<float*>(ctl_gen + 256);  // [TN]: 1 / (weight scale * token scale)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -369,7 +369,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(ctl.full + 8 * s, 1);
-            ptx::mbar_init(ctl.aready + 8 * s, kWorkerWarps);
+            ptx::mbar_init(ctl.aready + 8 * s, kPfWorkerWarps);
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
         ptx::mbar_init(ctl.accum, 1);
@@ -392,11 +392,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // ---------------- TMA producer: activation tile + plane words of the stage
         if (lane == 0) {
             bool ok = true;
-            int issued = 0;
+            int issued = 0, s = 0;
+            uint32_t ph = 0;
             const uint32_t tx = L::kBBytes + (uint32_t)p.q * L::kPlaneBytes;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+            for (int it = 0; it < iters; ++it) {
                 const int kb = kb_begin + it;
                 ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                 if (!ok) break;
@@ -408,6 +407,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 else
                     ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, m0 >> 5, kb * kBlockK, 0, ctl.full + 8 * s);
                 issued = it + 1;
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
             if (!ok)  // giving up: let the copies already issued land before the CTA exits
                 for (int it = max(0, issued - STAGES); it < issued; ++it)
@@ -417,9 +417,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // ---------------- UMMA issuer
         if (lane == 0) {
             bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < iters; ++it) {
                 ok = wait_bar(ctl.full + 8 * s, ph, ctl, 3) && wait_bar(ctl.aready + 8 * s, ph, ctl, 4);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
@@ -433,6 +433,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     ptx::umma_bf16(tmem_base, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
                 }
                 ptx::umma_commit(ctl.empty + 8 * s);
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
             if (ok) {
                 ptx::umma_commit(ctl.accum);
@@ -443,61 +444,72 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         }
     } else {
         // ---------------- workers: expansion, then epilogue
-        const int wid = warp - kWorkerWarp0;  // 0..7
+        const int wid = warp - kWorkerWarp0;  // 0..15
+        const int e = wid * 32 + lane;        // 0..511
         const long long plane_alpha = (long long)p.d_out * p.G;
 
         // power of two for the weights: q * max|alpha| lands in [2^13, 2^14)
         const float amax = __uint_as_float(__ldg(&p.hdr->alpha_max_bits));
         const int wsh = shift_for(exponent_of_bits(__float_as_uint(amax * (float)p.q)), 13);
         const float wscale = pow2f(wsh);
-        const float winv = pow2f(-wsh);
+        {
+            const float winv = pow2f(-wsh);
+            for (int i = e; i < TN; i += kPfWorkers)
+                out_scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
+        }
 
         Lut lut = {0u, 0u, 0u, 0u};
         int lut_key = -2;
         bool ok = true;
+        int s = 0;
+        uint32_t ph = 0;
 
         if (MODE == MODE_FWD) {
-            // task = (weight row, 32-wide half of the stage's 64 k).  The two halves of a row sit
-            // in adjacent lanes, so their scale loads coalesce.  The row's scales change only when
-            // k crosses a group boundary: the set for the next group is loaded when the current
-            // one is taken into use.
-            const int row = wid * 16 + (lane >> 1);
-            const int half = lane & 1;
+            // task = (weight row, 16 of the stage's 64 k).  The four tasks of a row sit in adjacent
+            // lanes, so their scale loads coalesce.  A row's scales change only when k crosses a
+            // group boundary: the set for the following group is requested when the current one is
+            // taken into use.
+            const int row = wid * 8 + (lane >> 2);
+            const int piece = lane & 3;
             const int j = m0 + row;
             const bool valid = j < p.d_out;
-            const uint32_t line_off = row * 128, lx = row & 7, chunk0 = half * 4;
+            const uint32_t line_off = row * 128, lx = row & 7, chunk0 = piece * 2;
+            const uint32_t bit_shift = (piece & 1) * 16;
+            const uint32_t word_off = row * 16 + ((piece >> 1) << 2);
             const int cstep = max(1, kBlockK / p.g);
-            auto group_of = [&](int kb) { return min((kb * kBlockK + half * 32) / p.g, p.G - 1); };
             AlphaSet<QM> cur, nxt;
-            int c_cur = (iters > 0) ? group_of(kb_begin) : 0;
+            int k_pos = kb_begin * kBlockK + piece * 16;
+            int c_cur = min(k_pos / p.g, p.G - 1);
+            int k_next = (c_cur + 1) * p.g;  // first k of the following group
             load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
             load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
-            for (int it = 0; it < iters; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+            for (int it = 0; it < iters; ++it, k_pos += kBlockK) {
                 const int kb = kb_begin + it;
-                const int c = group_of(kb);
-                if (c != c_cur) {
+                if (k_pos >= k_next && c_cur < p.G - 1) {
+                    c_cur = min(k_pos / p.g, p.G - 1);
+                    k_next = (c_cur + 1) * p.g;
                     cur = nxt;
-                    c_cur = c;
-                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c + cstep, p.G - 1), valid, wscale);
+                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
                 }
                 ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // plane words of the stage have landed
                 if (!ok) break;
                 const uint32_t st = smem_base + s * kStageBytes;
-                expand_task<QM>(cur, st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2), L::kPlaneBytes, lut,
+                expand_task<QM>(cur, st + L::kBitsOff + word_off + ((kb & 1) << 3), L::kPlaneBytes, bit_shift, lut,
                                 lut_key, p.q, st + line_off, lx, chunk0);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         } else {
-            // task = (K index j = 64*kb + jl, 32-wide quarter of the tile's 128 k).  Rows change with
-            // every stage, so the scales are fetched kPrefetch stages ahead.
-            const int jl = wid * 8 + (lane >> 2);
-            const int part = lane & 3;
-            const uint32_t line_off = ((part >> 1) * 8192) + jl * 128, lx = jl & 7, chunk0 = (part & 1) * 4;
-            const int c = min((m0 + part * 32) / p.g, p.G - 1);
+            // task = (K index j = 64*kb + jl, 16 of the tile's 128 k).  Rows change with every stage,
+            // so the scales are requested kPrefetch stages ahead.
+            const int jl = wid * 4 + (lane >> 3);
+            const int sub = lane & 7;
+            const uint32_t line_off = ((sub >> 2) * 8192) + jl * 128, lx = jl & 7, chunk0 = (sub & 3) * 2;
+            const uint32_t bit_shift = (sub & 1) * 16;
+            const uint32_t word_off = jl * 16 + ((sub >> 1) << 2);
+            const int c = min((m0 + sub * 16) / p.g, p.G - 1);
             AlphaSet<QM> ring[kPrefetch];
             auto fetch = [&](AlphaSet<QM>& slot, int kb) {
                 const int j = kb * kBlockK + jl;
@@ -511,32 +523,33 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 for (int d = 0; d < kPrefetch; ++d) {
                     const int it = it0 + d;
                     if (it < iters && ok) {
-                        const int s = it % STAGES;
-                        const uint32_t ph = (it / STAGES) & 1;
                         const AlphaSet<QM> cur = ring[d];
                         if (it + kPrefetch < iters) fetch(ring[d], kb_begin + it + kPrefetch);
                         ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);
                         if (ok) {
                             const uint32_t st = smem_base + s * kStageBytes;
-                            expand_task<QM>(cur, st + L::kBitsOff + jl * 16 + (part << 2), L::kPlaneBytes, lut, lut_key,
+                            expand_task<QM>(cur, st + L::kBitsOff + word_off, L::kPlaneBytes, bit_shift, lut, lut_key,
                                             p.q, st + line_off, lx, chunk0);
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                            if (++s == STAGES) { s = 0; ph ^= 1u; }
                         }
                     }
                 }
             }
         }
 
-        // epilogue: D[row, col] -> out[t0 + col][m0 + row]; warp w reads TMEM lanes 32*(w%4)..
+        // epilogue: D[row, col] -> out[t0 + col][m0 + row]; warp w reads TMEM lanes 32*(w%4).., the
+        // four warps that share a lane quarter take a quarter of the columns each
+        asm volatile("bar.sync 1, %0;" ::"n"(kPfWorkers) : "memory");  // out_scale written by all workers
         if (ok) ok = wait_bar(ctl.accum, 0, ctl, 7);
         if (ok) {
             ptx::tc_fence_after_sync();
             const int quarter = warp & 3;
-            const int half = wid >> 2;
-            constexpr int HN = TN / 2;
-            constexpr int CH = 16;
+            const int cq = wid >> 2;
+            constexpr int QN = TN / 4;
+            constexpr int CH = QN < 16 ? 8 : 16;
             int m = m0 + quarter * 32 + lane;
             if (MODE == MODE_BWDX) {
                 // accumulator row r holds k = 8*(r/8) + {0,4,1,5,2,6,3,7}[r % 8]
@@ -547,18 +560,22 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const float bias =
                 (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m_ok) ? __ldg(p.bias + m) : 0.0f;
 #pragma unroll 1
-            for (int cb = 0; cb < HN; cb += CH) {
-                const int col = half * HN + cb;
+            for (int cb = 0; cb < QN; cb += CH) {
+                const int col = cq * QN + cb;
                 if (t0 + col >= p.n) break;  // uniform in the warp
                 uint32_t v[CH];
-                ptx::tmem_ld_x16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col, v);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col;
+                if (CH == 8)
+                    ptx::tmem_ld_x8(taddr, v);
+                else
+                    ptx::tmem_ld_x16(taddr, v);
                 ptx::tmem_ld_wait();
                 if (m_ok) {
 #pragma unroll
                     for (int cidx = 0; cidx < CH; ++cidx) {
                         const int t = t0 + col + cidx;
                         if (t < p.n) {
-                            const float val = __uint_as_float(v[cidx]) * (winv * __ldg(p.tok_inv_scale + t));
+                            const float val = __uint_as_float(v[cidx]) * out_scale[col + cidx];
                             if (p.splits > 1) {
                                 p.partial[((long long)blockIdx.z * p.n + t) * p.Mdim + m] = val;
                             } else if (p.out_bf16) {
@@ -813,8 +830,10 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams 
                     ok = wait_bar(ctl.full + 8 * s, ph, ctl, 23);
                     if (ok) {
                         const uint32_t st = smem_base + s * kStageBytes;
-                        expand_task<QM>(cur, st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2), L::kPlaneBytes,
-                                        lut, lut_key, p.q, st + row * 128, lx, half * 4);
+                        const uint32_t baddr = st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2);
+                        expand_task<QM>(cur, baddr, L::kPlaneBytes, 0u, lut, lut_key, p.q, st + row * 128, lx, half * 4);
+                        expand_task<QM>(cur, baddr, L::kPlaneBytes, 16u, lut, lut_key, p.q, st + row * 128, lx,
+                                        half * 4 + 2);
                         if (x_task) {
                             const uint32_t xs[4] = {xcur.x, xcur.y, xcur.z, xcur.w};
                             float f[8];
@@ -938,7 +957,7 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
-constexpr size_t kSmemBudget = 232448 - 1024 - 512;  // 227 KiB minus alignment slack and the control block
+constexpr size_t kSmemBudget = 232448 - 1024 - 1280;  // 227 KiB minus alignment slack and the control block
 
 template <int MODE, int TN, int QM>
 constexpr int stages_for() {
@@ -949,7 +968,7 @@ constexpr int stages_for() {
 
 template <int MODE, int TN, int QM>
 constexpr size_t smem_for() {
-    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + 512;
+    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + 1280;
 }
 
 template <int MODE, int TN, int QM>
@@ -959,7 +978,8 @@ bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tm_bits, cons
     constexpr size_t smem = smem_for<MODE, TN, QM>();
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.n_tiles, (unsigned)pl.splits);
-    kern<<<grid, kThreads, smem, stream>>>(tm, tm_bits, p);
+    kern<<<grid, kPfThreads, smem, stream>>>(tm, tm_bits, p);
+    bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
 }
@@ -1006,6 +1026,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     if (ablocks > 128) ablocks = 128;
     if (ablocks < 1) ablocks = 1;
     prepare_kernel<<<(unsigned)(n + ablocks), 256, 0, s>>>(pp);
+    bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
 
     ExpandParams p;
@@ -1027,6 +1048,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
         const long long total = (long long)n * Mdim;
         splitk_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
             n, Mdim, pl.splits, p.partial, bias, out, (long long)ldo, p.out_bf16);
+    bcq::count_launch();
         BCQ_CUDA_TRY(cudaGetLastError());
     }
     return BCQ_OK;
@@ -1040,6 +1062,7 @@ bcq_status launch_decode(const CUtensorMap& tm_bits, const DecodeParams& p, cons
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.splits);
     kern<<<grid, kThreads, smem, s>>>(tm_bits, p);
+    bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
 }
@@ -1074,6 +1097,7 @@ bcq_status run_decode(int d_out, int d_in, int q, int g, int n, const void* X, s
         const long long total = (long long)n * d_out;
         splitk_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
             n, d_out, pl.splits, p.partial, bias, Y, (long long)ldy, p.out_bf16);
+    bcq::count_launch();
         BCQ_CUDA_TRY(cudaGetLastError());
     }
     return BCQ_OK;

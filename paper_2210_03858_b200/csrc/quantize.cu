@@ -251,6 +251,7 @@ cudaError_t launch_quantize(const QuantParams& p, cudaStream_t stream) {
         quantize_kernel<EPT, TW, true><<<(unsigned)blocks, threads, 0, stream>>>(p);
     else
         quantize_kernel<EPT, TW, false><<<(unsigned)blocks, threads, 0, stream>>>(p);
+    bcq::count_launch();
     return cudaGetLastError();
 }
 
@@ -318,6 +319,7 @@ extern "C" bcq_status bcq_dequantize(int d_out, int d_in, int q, int g, const ui
     dequantize_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
         d_out, d_in, q, g, (int)bcq_num_groups(d_in, g), (int)bcq_pitch_words(d_in), bits, alpha,
         W_hat, (long long)ldw);
+    bcq::count_launch();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return bcq::cuda_fail(e);
     return BCQ_OK;
