@@ -130,6 +130,34 @@ bcq_status bcq_linear_decode(int d_out, int d_in, int q, int g, int n, const voi
                              void* Y, size_t ldy, int y_dtype, void* ws, size_t ws_bytes,
                              void* stream);
 
+/* bcq_linear_decode without a caller-provided workspace.  (The paper has no counterpart; this is
+ * a convenience of the library.)
+ *
+ * Some callers of the decode path cannot hand over scratch memory: code that runs where
+ * cudaMalloc is off limits -- inside a region that must not touch the allocator (a latency-critical
+ * serving loop, a plugin that is only given its input and output tensors), or a process whose
+ * memory was carved up in advance.  For them the partial sums of the split over d_in live in a
+ * fixed array inside the library, BCQ_NOALLOC_SCRATCH_BYTES (2 MiB) of device memory that
+ * every GPU using the library holds from the moment the library is loaded until the process exits.
+ * The call allocates nothing and frees nothing.
+ *
+ *   - Same arguments and results as bcq_linear_decode, minus ws / ws_bytes.
+ *   - If bcq_workspace_bytes(BCQ_OP_DECODE, ...) for the shape exceeds
+ *     BCQ_NOALLOC_SCRATCH_BYTES the call returns BCQ_ERR_WORKSPACE and launches nothing (on a
+ *     B200 that is roughly n * d_out beyond 128K with a split d_in, e.g. 16 tokens of a
+ *     12288-row layer; 8 tokens of it fit).  Such problems need bcq_linear_decode.
+ *   - The first call on each device looks up the device address of the array
+ *     (cudaGetSymbolAddress) with that device current; make that first call outside any stream
+ *     capture.  Later calls on the device only launch kernels.
+ *   - All calls on a device share the one array.  It keeps whatever the last call left in it;
+ *     every call overwrites the part it reads, so nothing has to be cleared.  Two calls that may
+ *     overlap on the GPU (different streams, no dependency) race on it: serialise them. */
+#define BCQ_NOALLOC_SCRATCH_BYTES (2u << 20)
+bcq_status bcq_linear_decode_noalloc(int d_out, int d_in, int q, int g, int n, const void* X,
+                                     size_t ldx, const uint32_t* bits, const float* alpha,
+                                     const float* bias, void* Y, size_t ldy, int y_dtype,
+                                     void* stream);
+
 /* Input gradient (Eq. 3):  dX[t][k] = sum_j dY[t][j] * W_hat[j][k],  W_hat as in Eq. 1.
  *   dY in : bf16 [n][lddy];   dX out: dx_dtype [n][lddx], lddx >= d_in. */
 bcq_status bcq_linear_bwd_x(int d_out, int d_in, int q, int g, int n, const void* dY, size_t lddy,

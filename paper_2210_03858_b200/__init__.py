@@ -24,7 +24,7 @@ SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_cou
            "bcq_payload_bits", "bcq_workspace_bytes", "bcq_quantize", "bcq_dequantize",
            "bcq_linear_fwd", "bcq_linear_decode", "bcq_linear_bwd_x", "bcq_linear_bwd_alpha",
            "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag",
-           "bcq_kernel_launches")
+           "bcq_kernel_launches", "bcq_linear_decode_noalloc")
 
 
 class BcqError(RuntimeError):
@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
         l.bcq_linear_fwd.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_decode.restype = i
         l.bcq_linear_decode.argtypes = l.bcq_linear_fwd.argtypes
+        l.bcq_linear_decode_noalloc.restype = i
+        l.bcq_linear_decode_noalloc.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, vp, sz, i, vp]
         l.bcq_linear_bwd_x.restype = i
         l.bcq_linear_bwd_x.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_bwd_alpha.restype = i
@@ -197,6 +199,26 @@ def linear_decode(X, bits, alpha, d_in: int, g: int, bias=None, out=None, out_dt
     """bcq_linear_decode: same as linear_fwd for 1..16 tokens."""
     return _fwd(lib().bcq_linear_decode, OP_DECODE, "bcq_linear_decode", X, bits, alpha, d_in, g,
                 bias, out, out_dtype, ws)
+
+
+NOALLOC_SCRATCH_BYTES = 2 << 20
+
+
+def linear_decode_noalloc(X, bits, alpha, d_in: int, g: int, bias=None, out=None):
+    """bcq_linear_decode_noalloc: decode for callers that cannot provide scratch memory -- the
+    library call itself allocates nothing (its partial sums go to a fixed 2 MiB array inside the
+    library).  ``out`` must be given by such a caller; it is created here only as a convenience
+    for tests."""
+    torch = _torch()
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    q, d_out, _ = bits.shape
+    n = X.shape[0]
+    if out is None:
+        out = torch.empty((n, d_out), dtype=torch.float32, device=X.device)
+    _check(lib().bcq_linear_decode_noalloc(d_out, d_in, q, g, n, _ptr(X), X.stride(0), _ptr(bits),
+                                           _ptr(alpha), _ptr(bias), _ptr(out), out.stride(0),
+                                           _dtype_code(out), _stream()), "bcq_linear_decode_noalloc")
+    return out
 
 
 def linear_bwd_x(dY, bits, alpha, d_in: int, g: int, out=None, out_dtype=None, ws=None):

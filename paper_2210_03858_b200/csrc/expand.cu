@@ -26,6 +26,8 @@
 //     0,4,1,5,2,6,3,7 (that is what one PRMT pair produces).  For the forward the pre-pass writes
 //     the activations in the same order; for dX, where k indexes accumulator rows, the epilogue
 //     maps rows back.
+#include <mutex>
+
 #include "gemm_common.cuh"
 
 namespace {
@@ -1152,6 +1154,53 @@ extern "C" bcq_status bcq_linear_decode(int d_out, int d_in, int q, int g, int n
                                         size_t ws_bytes, void* stream) {
     return fwd_common(1, d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes,
                       stream);
+}
+
+// ------------------------------------------------------------------------------------------
+// decode without a caller-provided workspace
+// ------------------------------------------------------------------------------------------
+
+namespace {
+
+// Scratch for the split-K partial sums of bcq_linear_decode_noalloc.  Lives in every CUDA context
+// that loads this library.  In host code the symbol is only a handle: the device address comes
+// from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[BCQ_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+
+bcq_status noalloc_scratch_address(void** out) {
+    static void* address[kMaxDevices] = {};
+    static std::mutex lock;
+    int dev = -1;
+    BCQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return BCQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> guard(lock);
+    if (address[dev] == nullptr) {
+        void* p = nullptr;
+        BCQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        address[dev] = p;
+    }
+    *out = address[dev];
+    return BCQ_OK;
+}
+
+}  // namespace
+
+extern "C" bcq_status bcq_linear_decode_noalloc(int d_out, int d_in, int q, int g, int n, const void* X,
+                                                size_t ldx, const uint32_t* bits, const float* alpha,
+                                                const float* bias, void* Y, size_t ldy, int y_dtype,
+                                                void* stream) {
+    // validate first, so that a bad call neither touches the device nor resolves the symbol
+    bcq_status st = check_shape(d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1 || n > 16) return BCQ_ERR_SHAPE;
+    if (bcq::decode_workspace_bytes(d_out, d_in, q, g, n) > (size_t)BCQ_NOALLOC_SCRATCH_BYTES)
+        return BCQ_ERR_WORKSPACE;
+    void* scratch = nullptr;
+    if ((st = noalloc_scratch_address(&scratch)) != BCQ_OK) return st;
+    return fwd_common(1, d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, scratch,
+                      (size_t)BCQ_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 extern "C" bcq_status bcq_linear_bwd_x(int d_out, int d_in, int q, int g, int n, const void* dY,
