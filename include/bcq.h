@@ -116,8 +116,10 @@ bcq_status bcq_dequantize(int d_out, int d_in, int q, int g, const uint32_t* bit
  *   bias in : float [d_out] or NULL (the frozen bias of the layer)
  *   Y    out: y_dtype [n][ldy], ldy >= d_out
  *   ws      : scratch of bcq_workspace_bytes(BCQ_OP_FWD, ...) bytes, 16-byte aligned (NULL if 0)
- * Products are bf16 x bf16 accumulated in fp32; the scaled weight sum_i alpha_i b_i enters
- * the tensor core rounded to bf16. */
+ * Arithmetic: the scaled weight sum_i alpha_i b_i is formed in fp32 and rounded once to fp16;
+ * the bf16 activations are converted exactly to fp16 after a per-token power-of-two scaling
+ * that is undone on output; products are accumulated in fp32 in the tensor core.  The same
+ * holds for bcq_linear_decode and bcq_linear_bwd_x. */
 bcq_status bcq_linear_fwd(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
                           const uint32_t* bits, const float* alpha, const float* bias, void* Y,
                           size_t ldy, int y_dtype, void* ws, size_t ws_bytes, void* stream);
