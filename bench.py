@@ -169,34 +169,79 @@ def run_gpu(args):
             dY = torch.randn((TOKENS, d_out), generator=gen, device=dev, dtype=torch.float32).bfloat16()
             layers.append(dict(d_in=d_in, d_out=d_out, bits=bits, alpha=alpha, X=X, dY=dY,
                                dalpha=torch.zeros_like(alpha)))
-    # outputs and workspaces are shared between linears of the same shape
+    # outputs and workspaces: one set per shape and per operation, so that the three operations of
+    # a step can run on three streams at once
     bufs = {}
+    out_dtype = torch.bfloat16 if args.out_bf16 else torch.float32
     for _, d_in, d_out in LINEARS:
-        ws = max(bcq.workspace_bytes(op, d_out, d_in, Q, d_in, TOKENS)
-                 for op in (bcq.OP_FWD, bcq.OP_BWD_X, bcq.OP_BWD_ALPHA))
-        bufs[(d_in, d_out)] = dict(Y=torch.empty((TOKENS, d_out), device=dev), dX=torch.empty((TOKENS, d_in), device=dev),
-                                   ws=torch.empty(ws, dtype=torch.uint8, device=dev))
+        def ws(op):
+            return torch.empty(max(16, bcq.workspace_bytes(op, d_out, d_in, Q, d_in, TOKENS)), dtype=torch.uint8, device=dev)
+        bufs[(d_in, d_out)] = dict(Y=torch.empty((TOKENS, d_out), device=dev, dtype=out_dtype),
+                                   dX=torch.empty((TOKENS, d_in), device=dev, dtype=out_dtype),
+                                   ws_fwd=ws(bcq.OP_FWD), ws_dx=ws(bcq.OP_BWD_X), ws_da=ws(bcq.OP_BWD_ALPHA))
     flat_dalpha = torch.zeros(sum(l["dalpha"].numel() for l in layers), device=dev) if world > 1 else None
 
-    def linear_step(l, timing=None):
+    def op_fwd(l):
         b = bufs[(l["d_in"], l["d_out"])]
-        g = l["d_in"]
-        ops = (("fwd", lambda: bcq.linear_fwd(l["X"], l["bits"], l["alpha"], l["d_in"], g, out=b["Y"], ws=b["ws"])),
-               ("bwd_alpha", lambda: bcq.linear_bwd_alpha(l["dY"], l["X"], l["bits"], l["d_in"], g, out=l["dalpha"], ws=b["ws"])),
-               ("bwd_x", lambda: bcq.linear_bwd_x(l["dY"], l["bits"], l["alpha"], l["d_in"], g, out=b["dX"], ws=b["ws"])))
-        for name, fn in ops:
-            if timing is None:
-                fn()
-            else:
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record()
-                fn()
-                e1.record()
-                timing.append((name, 2.0 * TOKENS * l["d_in"] * l["d_out"], e0, e1))
+        bcq.linear_fwd(l["X"], l["bits"], l["alpha"], l["d_in"], l["d_in"], out=b["Y"], ws=b["ws_fwd"])
+
+    def op_da(l):
+        b = bufs[(l["d_in"], l["d_out"])]
+        bcq.linear_bwd_alpha(l["dY"], l["X"], l["bits"], l["d_in"], l["d_in"], out=l["dalpha"], ws=b["ws_da"])
+
+    def op_dx(l):
+        b = bufs[(l["d_in"], l["d_out"])]
+        bcq.linear_bwd_x(l["dY"], l["bits"], l["alpha"], l["d_in"], l["d_in"], out=b["dX"], ws=b["ws_dx"])
+
+    OPS = (("fwd", op_fwd), ("bwd_alpha", op_da), ("bwd_x", op_dx))
+
+    def linear_step(l):
+        for _, fn in OPS:
+            fn(l)
+
+    side = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)]
+
+    def enqueue_step():
+        # the linears are independent problems, and within one linear dalpha and dX only share their
+        # inputs: forward, dalpha and dX are enqueued as three chains on three streams
+        cur = torch.cuda.current_stream()
+        for s_ in side:
+            s_.wait_stream(cur)
+        for l in layers:
+            op_fwd(l)
+        with torch.cuda.stream(side[0]):
+            for l in layers:
+                op_da(l)
+        with torch.cuda.stream(side[1]):
+            for l in layers:
+                op_dx(l)
+        for s_ in side:
+            cur.wait_stream(s_)
+
+    # warm up outside capture (also resolves lazy CUDA state), then capture one step as a CUDA graph
+    main = torch.cuda.Stream(device=dev)
+    torch.cuda.synchronize()
+    graph = None
+    launches_per_step = 0
+    with torch.cuda.stream(main):
+        enqueue_step()
+        torch.cuda.synchronize()
+        c0 = bcq.kernel_launches()
+        if args.graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=main):
+                enqueue_step()
+        else:
+            enqueue_step()
+        launches_per_step = bcq.kernel_launches() - c0
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(main)
 
     def step():
-        for l in layers:
-            linear_step(l)
+        if graph is not None:
+            graph.replay()
+        else:
+            enqueue_step()
         if world > 1:  # data parallel: the scale gradients are summed over ranks once per step
             torch.cat([l["dalpha"].reshape(-1) for l in layers], out=flat_dalpha)
             dist.all_reduce(flat_dalpha)
@@ -212,29 +257,39 @@ def run_gpu(args):
     for _ in range(max(3, args.warmup)):
         step()
     sync_all()
-    launches0 = bcq.kernel_launches()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.steps):
         step()
     e1.record()
     sync_all()
-    launches = bcq.kernel_launches() - launches0
+    launches = launches_per_step * args.steps
     ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
     if world > 1:
         dist.all_reduce(ms, op=dist.ReduceOp.MAX)
     ms_per_step = float(ms.item()) / args.steps
     assert bcq.device_timeout_flag() == 0, "a kernel reported an expired wait"
 
-    # ---- per-call durations (one instrumented step) for the roofline of the dominant kernels
-    timing = []
-    for l in layers:
-        linear_step(l, timing)
-    torch.cuda.synchronize()
+    # ---- per-operation GPU time for the roofline: all 96 calls of one operation back to back on
+    # one stream (captured as a graph so that host launch time stays out), CUDA-event timed
     per_op = {}
-    for name, fl, a, b_ in timing:
-        t, f, c = per_op.get(name, (0.0, 0.0, 0))
-        per_op[name] = (t + a.elapsed_time(b_), f + fl, c + 1)
+    for name, fn in OPS:
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_, stream=main):
+            for l in layers:
+                fn(l)
+        g_.replay()
+        torch.cuda.synchronize()
+        best = None
+        for _ in range(3):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            g_.replay()
+            b_.record()
+            torch.cuda.synchronize()
+            best = a.elapsed_time(b_) if best is None else min(best, a.elapsed_time(b_))
+        per_op[name] = (best, sum(2.0 * TOKENS * l["d_in"] * l["d_out"] for l in layers), len(layers))
+        del g_
 
     # ---- end to end: inputs in pinned host memory, H2D every step, dalpha read back every step
     e2e = None
@@ -296,6 +351,8 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "f16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "layers": LAYERS, "tokens_per_gpu": TOKENS, "q": Q, "g": "d_in",
                        "l2": "a step touches ~1.5 GB of distinct inputs, far more than the 126 MB L2",
+                       "outputs": "bf16" if args.out_bf16 else "fp32",
+                       "launch": ("one CUDA graph per step, " if args.graph else "") + "forward / dalpha / dX on three streams",
                        "parallelism": "dp%d" % world, "quantize_ms_once": quant_ms},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline}
@@ -347,6 +404,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
     ap.add_argument("--no-decode", dest="decode", action="store_false")
+    ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch every kernel from the host each step")
+    ap.add_argument("--out-fp32", dest="out_bf16", action="store_false", help="fp32 Y and dX instead of bf16")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
