@@ -135,6 +135,50 @@ __device__ __forceinline__ void expand16_lut(uint32_t w0, uint32_t w1, uint32_t 
         ptx::st_shared_v4(line + (((chunk0 + u) ^ lx) << 4), R[0][u], R[1][u], R[2][u], R[3][u]);
 }
 
+// 32 weights (whole plane words): the selector word S of residue r serves both halves, low 16 bits
+// for weights 0..15 and high 16 bits for weights 16..31.  Four chunks, slots chunk0..chunk0+3.
+template <bool Q4>
+__device__ __forceinline__ void expand32_lut(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
+                                             const Lut& t, uint32_t line, uint32_t lx, uint32_t chunk0) {
+    uint32_t x0 = w0, x1 = w1, x2 = w2, nf = 0u;
+    if (Q4) {
+        nf = ~w3;
+        x0 = ~(w0 ^ w3);
+        x1 = ~(w1 ^ w3);
+        x2 = ~(w2 ^ w3);
+    }
+    constexpr uint32_t M = 0x11111111u;
+    uint32_t R[4][2][2];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const uint32_t a = x0 >> r;
+        const uint32_t b = (r >= 1) ? (x1 >> (r >= 1 ? r - 1 : 0)) : (x1 << 1);
+        const uint32_t c = (r >= 2) ? (x2 >> (r >= 2 ? r - 2 : 0)) : (x2 << (r >= 2 ? 0 : 2 - r));
+        const uint32_t S = (a & M) | (b & (M << 1)) | (c & (M << 2));
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t sel = h ? (S >> 16) : S;  // weights 16h + 4m + r, m = 0..3
+            uint32_t hb = prmt(t.th0, t.th1, sel);
+            const uint32_t lb = prmt(t.tl0, t.tl1, sel);
+            if (Q4) {
+                const int p0 = 16 * h + r;  // bit of weight m = 0; m = 2 is 8 bits up, m = 1, 3 are 4 bits up
+                const uint32_t s02 = (p0 <= 7) ? (nf << (p0 <= 7 ? 7 - p0 : 0)) : (nf >> (p0 > 7 ? p0 - 7 : 0));
+                const uint32_t s13 = (p0 <= 3) ? (nf << (p0 <= 3 ? 3 - p0 : 0)) : (nf >> (p0 > 3 ? p0 - 3 : 0));
+                const uint32_t flip = prmt(s02, s13, 0xD9C8u);
+                hb ^= flip & 0x80808080u;
+            }
+            R[r][h][0] = prmt(lb, hb, 0x5140u);
+            R[r][h][1] = prmt(lb, hb, 0x7362u);
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            ptx::st_shared_v4(line + (((chunk0 + 2 * h + u) ^ lx) << 4), R[0][h][u], R[1][h][u], R[2][h][u],
+                              R[3][h][u]);
+}
+
 // Same result through fp32 sums, any q <= 8.  w[i] = plane words (bits 0..15 used), a[i] = scales.
 __device__ __forceinline__ void expand16_sum(const uint32_t (&w)[BCQ_MAX_Q], const float (&a)[BCQ_MAX_Q],
                                              int q, uint32_t line, uint32_t lx, uint32_t chunk0) {
@@ -208,14 +252,60 @@ __device__ __forceinline__ void expand_task(const AlphaSet<QM>& as, uint32_t bit
     }
 }
 
+// 32 weights (one whole plane word per plane): two 16-weight halves from one set of loads.
+template <int QM>
+__device__ __forceinline__ void expand_task32(const AlphaSet<QM>& as, uint32_t bits_addr, uint32_t plane_stride,
+                                              Lut& lut, int& lut_key, int q, uint32_t line, uint32_t lx,
+                                              uint32_t chunk0) {
+    uint32_t w[NumWords<QM>::value];
+#pragma unroll
+    for (int i = 0; i < NumWords<QM>::value; ++i)
+        w[i] = (i < q) ? ptx::ld_shared_u32(bits_addr + i * plane_stride) : 0u;
+    if (QM == QM_GENERIC) {
+        uint32_t w8[BCQ_MAX_Q];
+        float a8[BCQ_MAX_Q];
+#pragma unroll
+        for (int i = 0; i < BCQ_MAX_Q; ++i) {
+            w8[i] = w[i % NumWords<QM>::value];
+            a8[i] = as.a[i % NumWords<QM>::value];
+        }
+        expand16_sum(w8, a8, q, line, lx, chunk0);
+#pragma unroll
+        for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
+        expand16_sum(w8, a8, q, line, lx, chunk0 + 2);
+    } else {
+        if (as.key != lut_key) {
+            lut = (QM == QM_LUT4) ? build_lut(as.a[0], as.a[1], as.a[2], as.a[3])
+                                  : build_lut(as.a[0], as.a[1], as.a[2], 0.0f);
+            lut_key = as.key;
+        }
+        expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, line, lx, chunk0);
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // pre-pass: activations -> fp16 with a per-token power-of-two scale; max |alpha|
 // ------------------------------------------------------------------------------------------
 
+constexpr int kMaxAlphaBlocks = 124;
+
+// Head of the forward / dX workspace: max |alpha| of each pre-pass block that scanned alpha (bit
+// patterns; the consumer takes the maximum over the first `nblocks`).  No zero-initialisation.
 struct WsHeader {
-    uint32_t alpha_max_bits;  // bits of max |alpha| (atomicMax on the unsigned bit pattern)
+    uint32_t nblocks;
     uint32_t pad[3];
+    uint32_t block_max[kMaxAlphaBlocks];
 };
+
+// Power of two for the weights: q * max|alpha| lands in [2^13, 2^14).  Called by whole warps.
+__device__ __forceinline__ int weight_shift(const WsHeader* hdr, int q) {
+    const int nb = (int)__ldg(&hdr->nblocks);
+    uint32_t m = 0u;
+    for (int b = threadIdx.x & 31; b < nb; b += 32) m = max(m, __ldg(&hdr->block_max[b]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    return shift_for(exponent_of_bits(__float_as_uint(__uint_as_float(m) * (float)q)), 13);
+}
 
 struct PrepParams {
     int n, K, permute, act_blocks;
@@ -240,7 +330,14 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
             m = max(m, __float_as_uint(__ldg(p.alpha + i)) & 0x7FFFFFFFu);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (lane == 0 && m != 0u) atomicMax(&p.hdr->alpha_max_bits, m);
+        if (lane == 0) red[warp] = m;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int w = 0; w < 8; ++w) m = max(m, red[w]);
+            p.hdr->block_max[blockIdx.x - p.act_blocks] = m;
+            if ((int)blockIdx.x == p.act_blocks) p.hdr->nblocks = (uint32_t)nb;
+        }
         return;
     }
     // ---- one token row
@@ -303,9 +400,10 @@ struct ExpandParams {
     int num_kb;        // K blocks of 64 over d_in (fwd) or d_out (dX)
     int kb_per_split;
     int splits;
+    int m_tiles, n_tiles;
     const float* alpha;
     const float* bias;           // fwd only, may be null
-    const WsHeader* hdr;         // max |alpha|
+    const WsHeader* hdr;         // max |alpha| per pre-pass block
     const float* tok_inv_scale;  // [n]
     void* out;                   // [n][ldo]
     long long ldo;
@@ -327,11 +425,18 @@ struct StageLayout {
     static constexpr uint32_t kStageBytes = kBitsOff + kBitsBytes;
 };
 
-// Prefill kernels run 16 worker warps (plus the TMA and UMMA warps): a task is 16 weights of one
-// row, so that four warps per scheduler hide each other's dependency stalls.
+// Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
+// running at the same time share activation tiles in L2).  22 warps:
+//   warp 0        TMA producer (activation tile + plane words of each stage)
+//   warp 1        UMMA issuer, owner of the tensor-memory allocation (two accumulators)
+//   warps 2..17   workers in two groups of eight that take alternate pipeline stages; a task is
+//                 32 weights of one row, so a group rebuilds one 128 x 64 weight tile
+//   warps 18..21  epilogue: drain one accumulator while the main loop fills the other
 constexpr int kPfWorkerWarps = 16;
-constexpr int kPfWorkers = kPfWorkerWarps * 32;
-constexpr int kPfThreads = (kWorkerWarp0 + kPfWorkerWarps) * 32;
+constexpr int kPfGroupWarps = 8;
+constexpr int kPfEpiWarp0 = kWorkerWarp0 + kPfWorkerWarps;  // 18
+constexpr int kPfEpiWarps = 4;
+constexpr int kPfThreads = (kPfEpiWarp0 + kPfEpiWarps) * 32;  // 704
 
 template <int MODE, int TN, int STAGES, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
@@ -339,6 +444,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                    const ExpandParams p) {
     using L = StageLayout<MODE, TN, QM>;
     constexpr uint32_t kStageBytes = L::kStageBytes;
+    constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
     // fp16 x fp16 -> fp32; A is MN-major for dX
     constexpr uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
                                 ~((1u << 7) | (1u << 10));
@@ -353,28 +459,27 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     ctl.full = ctl_base;
     ctl.aready = ctl_base + 8 * STAGES;
     ctl.empty = ctl_base + 16 * STAGES;
-    ctl.accum = ctl_base + 24 * STAGES;
-    ctl.spare = ctl.accum + 8;
-    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 16);
-    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 20);
+    ctl.accum = ctl_base + 24 * STAGES;        // accumulator full [2]
+    const uint32_t acc_empty = ctl.accum + 16;  // accumulator drained [2]
+    ctl.spare = acc_empty + 16;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 40);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 44);
     ctl.device_flag = &g_timeout_flag;
-    float* out_scale = reinterpret_cast<float*>(ctl_gen + 256);  // [TN]: 1 / (weight scale * token scale)
+    float* out_scale = reinterpret_cast<float*>(ctl_gen + 256);  // [2][TN]: 1 / (weight scale * token scale)
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int m0 = blockIdx.x * kBlockM;
-    const int t0 = blockIdx.y * TN;
-    const int kb_begin = blockIdx.z * p.kb_per_split;
-    const int kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
-    const int iters = kb_end - kb_begin;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(ctl.full + 8 * s, 1);
-            ptx::mbar_init(ctl.aready + 8 * s, kPfWorkerWarps);
+            ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps);
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
-        ptx::mbar_init(ctl.accum, 1);
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(ctl.accum + 8 * a, 1);
+            ptx::mbar_init(acc_empty + 8 * a, kPfEpiWarps);
+        }
         ptx::mbar_init(ctl.spare, 1);
         *ctl.abort_flag = 0;
         ptx::fence_mbar_init();
@@ -382,7 +487,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         ptx::prefetch_tmap(&tmap_bits);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), TmemCols<TN>::value);
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
@@ -390,168 +495,201 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_holder;
 
+    // every role walks the same sequence of tiles and pipeline stages
+    const int num_tiles = p.m_tiles * p.n_tiles * p.splits;
+    auto tile_coords = [&](int tile, int& m0, int& t0, int& z, int& kb_begin, int& iters) {
+        const int mt = tile % p.m_tiles;
+        const int rest = tile / p.m_tiles;
+        m0 = mt * kBlockM;
+        t0 = (rest % p.n_tiles) * TN;
+        z = rest / p.n_tiles;
+        kb_begin = z * p.kb_per_split;
+        iters = min(p.num_kb, kb_begin + p.kb_per_split) - kb_begin;
+    };
+
     if (warp == 0) {
-        // ---------------- TMA producer: activation tile + plane words of the stage
+        // ---------------- TMA producer
         if (lane == 0) {
             bool ok = true;
-            int issued = 0, s = 0;
+            int s = 0, in_flight = 0;
             uint32_t ph = 0;
             const uint32_t tx = L::kBBytes + (uint32_t)p.q * L::kPlaneBytes;
-            for (int it = 0; it < iters; ++it) {
-                const int kb = kb_begin + it;
-                ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
-                if (!ok) break;
-                const uint32_t st = smem_base + s * kStageBytes;
-                ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, tx);
-                ptx::tma_load_2d(st + kABytes, &tmap_b, kb * kBlockK, t0, ctl.full + 8 * s);
-                if (MODE == MODE_FWD)
-                    ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, (kb >> 1) * 4, m0, 0, ctl.full + 8 * s);
-                else
-                    ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, m0 >> 5, kb * kBlockK, 0, ctl.full + 8 * s);
-                issued = it + 1;
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int m0, t0, z, kb_begin, iters;
+                tile_coords(tile, m0, t0, z, kb_begin, iters);
+                for (int it = 0; it < iters; ++it) {
+                    const int kb = kb_begin + it;
+                    ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
+                    if (!ok) break;
+                    const uint32_t st = smem_base + s * kStageBytes;
+                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, tx);
+                    ptx::tma_load_2d(st + kABytes, &tmap_b, kb * kBlockK, t0, ctl.full + 8 * s);
+                    if (MODE == MODE_FWD)
+                        ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, (kb >> 1) * 4, m0, 0, ctl.full + 8 * s);
+                    else
+                        ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, m0 >> 5, kb * kBlockK, 0, ctl.full + 8 * s);
+                    in_flight = min(in_flight + 1, STAGES);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
             }
-            if (!ok)  // giving up: let the copies already issued land before the CTA exits
-                for (int it = max(0, issued - STAGES); it < issued; ++it)
-                    wait_bar(ctl.full + 8 * (it % STAGES), (it / STAGES) & 1, ctl, 2);
+            if (!ok) {
+                // giving up: let the copies already issued land before the CTA exits.  The last
+                // `in_flight` stages before (s, ph) were issued with the phase they had then.
+                int bs = s;
+                uint32_t bph = ph;
+                for (int i = 0; i < in_flight; ++i) {
+                    if (bs == 0) { bs = STAGES; bph ^= 1u; }
+                    --bs;
+                    wait_bar(ctl.full + 8 * bs, bph, ctl, 2);
+                }
+            }
         }
     } else if (warp == 1) {
         // ---------------- UMMA issuer
         if (lane == 0) {
             bool ok = true;
-            int s = 0;
+            int s = 0, lt = 0;
             uint32_t ph = 0;
-            for (int it = 0; it < iters; ++it) {
-                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 3) && wait_bar(ctl.aready + 8 * s, ph, ctl, 4);
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+                int m0, t0, z, kb_begin, iters;
+                tile_coords(tile, m0, t0, z, kb_begin, iters);
+                const int acc = lt & 1;
+                const uint32_t acc_ph = (lt >> 1) & 1;
+                ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // epilogue has drained it
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t sa = smem_base + s * kStageBytes;
-                const uint32_t sb = sa + kABytes;
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * TmemCols<TN>::value;
+                for (int it = 0; it < iters; ++it) {
+                    ok = wait_bar(ctl.full + 8 * s, ph, ctl, 3) && wait_bar(ctl.aready + 8 * s, ph, ctl, 4);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t sa = smem_base + s * kStageBytes;
+                    const uint32_t sb = sa + kABytes;
 #pragma unroll
-                for (int kk = 0; kk < kBlockK / 16; ++kk) {
-                    const uint64_t da = (MODE == MODE_FWD) ? ptx::make_smem_desc(sa + kk * 32, 16, 1024)
-                                                           : ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
-                    const uint64_t db = ptx::make_smem_desc(sb + kk * 32, 16, 1024);
-                    ptx::umma_bf16(tmem_base, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBlockK / 16; ++kk) {
+                        const uint64_t da = (MODE == MODE_FWD) ? ptx::make_smem_desc(sa + kk * 32, 16, 1024)
+                                                               : ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
+                        const uint64_t db = ptx::make_smem_desc(sb + kk * 32, 16, 1024);
+                        ptx::umma_bf16(d_tmem, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    ptx::umma_commit(ctl.empty + 8 * s);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                ptx::umma_commit(ctl.empty + 8 * s);
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (ok) ptx::umma_commit(ctl.accum + 8 * acc);
             }
-            if (ok) {
-                ptx::umma_commit(ctl.accum);
-            } else {
+            if (!ok) {
                 ptx::umma_commit(ctl.spare);
                 wait_bar(ctl.spare, 0, ctl, 5);
             }
         }
-    } else {
-        // ---------------- workers: expansion, then epilogue
+    } else if (warp < kPfEpiWarp0) {
+        // ---------------- workers
         const int wid = warp - kWorkerWarp0;  // 0..15
-        const int e = wid * 32 + lane;        // 0..511
+        const int group = wid >> 3;           // takes the stages whose running index has this parity
+        const int wl = wid & 7;
         const long long plane_alpha = (long long)p.d_out * p.G;
-
-        // power of two for the weights: q * max|alpha| lands in [2^13, 2^14)
-        const float amax = __uint_as_float(__ldg(&p.hdr->alpha_max_bits));
-        const int wsh = shift_for(exponent_of_bits(__float_as_uint(amax * (float)p.q)), 13);
-        const float wscale = pow2f(wsh);
-        {
-            const float winv = pow2f(-wsh);
-            for (int i = e; i < TN; i += kPfWorkers)
-                out_scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
-        }
+        const float wscale = pow2f(weight_shift(p.hdr, p.q));
 
         Lut lut = {0u, 0u, 0u, 0u};
         int lut_key = -2;
         bool ok = true;
-        int s = 0;
+        int s = 0, gi = 0;  // stage slot and running stage index (its parity selects the group)
         uint32_t ph = 0;
 
-        if (MODE == MODE_FWD) {
-            // task = (weight row, 16 of the stage's 64 k).  The four tasks of a row sit in adjacent
-            // lanes, so their scale loads coalesce.  A row's scales change only when k crosses a
-            // group boundary: the set for the following group is requested when the current one is
-            // taken into use.
-            const int row = wid * 8 + (lane >> 2);
-            const int piece = lane & 3;
-            const int j = m0 + row;
-            const bool valid = j < p.d_out;
-            const uint32_t line_off = row * 128, lx = row & 7, chunk0 = piece * 2;
-            const uint32_t bit_shift = (piece & 1) * 16;
-            const uint32_t word_off = row * 16 + ((piece >> 1) << 2);
-            const int cstep = max(1, kBlockK / p.g);
-            AlphaSet<QM> cur, nxt;
-            int k_pos = kb_begin * kBlockK + piece * 16;
-            int c_cur = min(k_pos / p.g, p.G - 1);
-            int k_next = (c_cur + 1) * p.g;  // first k of the following group
-            load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
-            load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
-            for (int it = 0; it < iters; ++it, k_pos += kBlockK) {
-                const int kb = kb_begin + it;
-                if (k_pos >= k_next && c_cur < p.G - 1) {
-                    c_cur = min(k_pos / p.g, p.G - 1);
-                    k_next = (c_cur + 1) * p.g;
-                    cur = nxt;
-                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, min(c_cur + cstep, p.G - 1), valid, wscale);
-                }
-                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // plane words of the stage have landed
-                if (!ok) break;
-                const uint32_t st = smem_base + s * kStageBytes;
-                expand_task<QM>(cur, st + L::kBitsOff + word_off + ((kb & 1) << 3), L::kPlaneBytes, bit_shift, lut,
-                                lut_key, p.q, st + line_off, lx, chunk0);
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
-            }
-        } else {
-            // task = (K index j = 64*kb + jl, 16 of the tile's 128 k).  Rows change with every stage,
-            // so the scales are requested kPrefetch stages ahead.
-            const int jl = wid * 4 + (lane >> 3);
-            const int sub = lane & 7;
-            const uint32_t line_off = ((sub >> 2) * 8192) + jl * 128, lx = jl & 7, chunk0 = (sub & 3) * 2;
-            const uint32_t bit_shift = (sub & 1) * 16;
-            const uint32_t word_off = jl * 16 + ((sub >> 1) << 2);
-            const int c = min((m0 + sub * 16) / p.g, p.G - 1);
-            AlphaSet<QM> ring[kPrefetch];
-            auto fetch = [&](AlphaSet<QM>& slot, int kb) {
-                const int j = kb * kBlockK + jl;
-                load_alpha<QM>(slot, p.alpha, plane_alpha, p.G, p.q, j, c, j < p.d_out, wscale);
-            };
-#pragma unroll
-            for (int d = 0; d < kPrefetch; ++d)
-                if (d < iters) fetch(ring[d], kb_begin + d);
-            for (int it0 = 0; it0 < iters && ok; it0 += kPrefetch) {
-#pragma unroll
-                for (int d = 0; d < kPrefetch; ++d) {
-                    const int it = it0 + d;
-                    if (it < iters && ok) {
-                        const AlphaSet<QM> cur = ring[d];
-                        if (it + kPrefetch < iters) fetch(ring[d], kb_begin + it + kPrefetch);
-                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);
-                        if (ok) {
-                            const uint32_t st = smem_base + s * kStageBytes;
-                            expand_task<QM>(cur, st + L::kBitsOff + word_off, L::kPlaneBytes, bit_shift, lut, lut_key,
-                                            p.q, st + line_off, lx, chunk0);
-                            ptx::fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                            if (++s == STAGES) { s = 0; ph ^= 1u; }
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            int m0, t0, z, kb_begin, iters;
+            tile_coords(tile, m0, t0, z, kb_begin, iters);
+            if (MODE == MODE_FWD) {
+                // task = (weight row, 32-wide half of the stage's 64 k); the two halves of a row sit
+                // in adjacent lanes so that their scale loads coalesce.  The scales of the group that
+                // follows are requested when the current ones are taken into use.
+                const int row = wl * 16 + (lane >> 1);
+                const int half = lane & 1;
+                const int j = m0 + row;
+                const bool valid = j < p.d_out;
+                const uint32_t line_off = row * 128, lx = row & 7, chunk0 = half * 4;
+                const uint32_t word_off = row * 16 + (half << 2);
+                const int first = (gi & 1) == group ? 0 : 1;  // first stage of this tile that is ours
+                AlphaSet<QM> cur, nxt;
+                int c_cur = min(((kb_begin + first) * kBlockK + half * 32) / p.g, p.G - 1);
+                int c_nxt = min(c_cur + max(1, 2 * kBlockK / p.g), p.G - 1);
+                load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
+                load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c_nxt, valid, wscale);
+                for (int it = 0; it < iters; ++it, ++gi) {
+                    if ((gi & 1) == group) {
+                        const int kb = kb_begin + it;
+                        const int c = min((kb * kBlockK + half * 32) / p.g, p.G - 1);
+                        if (c != c_cur) {
+                            if (c == c_nxt) cur = nxt;
+                            else load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c, valid, wscale);
+                            c_cur = c;
+                            c_nxt = min(c + max(1, 2 * kBlockK / p.g), p.G - 1);
+                            load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c_nxt, valid, wscale);
                         }
+                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // plane words of the stage have landed
+                        if (!ok) break;
+                        const uint32_t st = smem_base + s * kStageBytes;
+                        expand_task32<QM>(cur, st + L::kBitsOff + word_off + ((kb & 1) << 3), L::kPlaneBytes, lut,
+                                          lut_key, p.q, st + line_off, lx, chunk0);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
                     }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            } else {
+                // task = (K index j = 64*kb + jl, 32-wide quarter of the tile's 128 k).  Rows change
+                // with every stage: the scales of our next stage are requested when the current ones
+                // are taken into use (two pipeline stages ahead).
+                const int jl = wl * 8 + (lane >> 2);
+                const int part = lane & 3;
+                const uint32_t line_off = ((part >> 1) * 8192) + jl * 128, lx = jl & 7, chunk0 = (part & 1) * 4;
+                const uint32_t word_off = jl * 16 + (part << 2);
+                const int c = min((m0 + part * 32) / p.g, p.G - 1);
+                const int first = (gi & 1) == group ? 0 : 1;
+                AlphaSet<QM> cur, nxt;
+                {
+                    const int j = (kb_begin + first) * kBlockK + jl;
+                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c, (first < iters) && (j < p.d_out), wscale);
+                }
+                for (int it = 0; it < iters; ++it, ++gi) {
+                    if ((gi & 1) == group) {
+                        cur = nxt;
+                        const int jn = (kb_begin + it + 2) * kBlockK + jl;
+                        load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, jn, c, (it + 2 < iters) && (jn < p.d_out), wscale);
+                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);
+                        if (!ok) break;
+                        const uint32_t st = smem_base + s * kStageBytes;
+                        expand_task32<QM>(cur, st + L::kBitsOff + word_off, L::kPlaneBytes, lut, lut_key, p.q,
+                                          st + line_off, lx, chunk0);
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                    }
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
         }
-
-        // epilogue: D[row, col] -> out[t0 + col][m0 + row]; warp w reads TMEM lanes 32*(w%4).., the
-        // four warps that share a lane quarter take a quarter of the columns each
-        asm volatile("bar.sync 1, %0;" ::"n"(kPfWorkers) : "memory");  // out_scale written by all workers
-        if (ok) ok = wait_bar(ctl.accum, 0, ctl, 7);
-        if (ok) {
+    } else {
+        // ---------------- epilogue warps: D[row, col] -> out[t0 + col][m0 + row]
+        const int ew = warp - kPfEpiWarp0;  // 0..3
+        const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
+        const int et = ew * 32 + lane;      // 0..127
+        const float winv = pow2f(-weight_shift(p.hdr, p.q));
+        bool ok = true;
+        int lt = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+            int m0, t0, z, kb_begin, iters;
+            tile_coords(tile, m0, t0, z, kb_begin, iters);
+            const int acc = lt & 1;
+            const uint32_t acc_ph = (lt >> 1) & 1;
+            float* scale = out_scale + acc * TN;
+            for (int i = et; i < TN; i += kPfEpiWarps * 32)
+                scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
+            asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
+            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7);
+            if (!ok) break;
             ptx::tc_fence_after_sync();
-            const int quarter = warp & 3;
-            const int cq = wid >> 2;
-            constexpr int QN = TN / 4;
-            constexpr int CH = QN < 16 ? 8 : 16;
             int m = m0 + quarter * 32 + lane;
             if (MODE == MODE_BWDX) {
                 // accumulator row r holds k = 8*(r/8) + {0,4,1,5,2,6,3,7}[r % 8]
@@ -561,25 +699,21 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const bool m_ok = m < p.Mdim;
             const float bias =
                 (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m_ok) ? __ldg(p.bias + m) : 0.0f;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
 #pragma unroll 1
-            for (int cb = 0; cb < QN; cb += CH) {
-                const int col = cq * QN + cb;
+            for (int col = 0; col < TN; col += 16) {
                 if (t0 + col >= p.n) break;  // uniform in the warp
-                uint32_t v[CH];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)col;
-                if (CH == 8)
-                    ptx::tmem_ld_x8(taddr, v);
-                else
-                    ptx::tmem_ld_x16(taddr, v);
+                uint32_t v[16];
+                ptx::tmem_ld_x16(t_row + (uint32_t)col, v);
                 ptx::tmem_ld_wait();
                 if (m_ok) {
 #pragma unroll
-                    for (int cidx = 0; cidx < CH; ++cidx) {
+                    for (int cidx = 0; cidx < 16; ++cidx) {
                         const int t = t0 + col + cidx;
                         if (t < p.n) {
-                            const float val = __uint_as_float(v[cidx]) * out_scale[col + cidx];
+                            const float val = __uint_as_float(v[cidx]) * scale[col + cidx];
                             if (p.splits > 1) {
-                                p.partial[((long long)blockIdx.z * p.n + t) * p.Mdim + m] = val;
+                                p.partial[((long long)z * p.n + t) * p.Mdim + m] = val;
                             } else if (p.out_bf16) {
                                 reinterpret_cast<__nv_bfloat16*>(p.out)[(long long)t * p.ldo + m] =
                                     __float2bfloat16_rn(val + bias);
@@ -590,6 +724,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     }
                 }
             }
+            // the accumulator (and this tile's scale row) may be reused
+            ptx::tc_fence_before_sync();
+            asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
+            if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * acc);
         }
     }
 
@@ -597,7 +735,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, TmemCols<TN>::value);
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -833,9 +971,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams 
                     if (ok) {
                         const uint32_t st = smem_base + s * kStageBytes;
                         const uint32_t baddr = st + L::kBitsOff + row * 16 + (((kb & 1) * 2 + half) << 2);
-                        expand_task<QM>(cur, baddr, L::kPlaneBytes, 0u, lut, lut_key, p.q, st + row * 128, lx, half * 4);
-                        expand_task<QM>(cur, baddr, L::kPlaneBytes, 16u, lut, lut_key, p.q, st + row * 128, lx,
-                                        half * 4 + 2);
+                        expand_task32<QM>(cur, baddr, L::kPlaneBytes, lut, lut_key, p.q, st + row * 128, lx, half * 4);
                         if (x_task) {
                             const uint32_t xs[4] = {xcur.x, xcur.y, xcur.z, xcur.w};
                             float f[8];
@@ -931,7 +1067,7 @@ ExpandPlan plan_expand(int Mdim, int Kdim, int n) {
     pl.kb_per_split = ceil_div(pl.num_kb, splits);
     pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
     pl.ld_act = (int)align_up((size_t)Kdim, 8);
-    pl.off_tok = sizeof(WsHeader);
+    pl.off_tok = align_up(sizeof(WsHeader), 128);
     pl.off_act = align_up(pl.off_tok + (size_t)n * sizeof(float), 128);
     pl.off_partial = align_up(pl.off_act + (size_t)n * pl.ld_act * 2, 128);
     pl.total = pl.off_partial + (pl.splits > 1 ? (size_t)pl.splits * n * Mdim * sizeof(float) : 0);
@@ -959,18 +1095,21 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
-constexpr size_t kSmemBudget = 232448 - 1024 - 1280;  // 227 KiB minus alignment slack and the control block
+constexpr size_t kCtlBytes = 256 + 2 * 256 * 4;     // barriers + two rows of output scales
+constexpr size_t kSmemBudget = 232448 - 1024 - kCtlBytes;  // 227 KiB minus alignment slack and the control block
 
 template <int MODE, int TN, int QM>
 constexpr int stages_for() {
     constexpr size_t per = StageLayout<MODE, TN, QM>::kStageBytes;
     constexpr int fit = (int)(kSmemBudget / per);
-    return fit > 6 ? 6 : fit;
+    // even, because the two worker groups alternate stages: with an even count a group meets the
+    // same slots in every round and never waits on a barrier phase it has not seen complete
+    return fit >= 6 ? 6 : (fit >= 4 ? 4 : 2);
 }
 
 template <int MODE, int TN, int QM>
 constexpr size_t smem_for() {
-    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + 1280;
+    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + kCtlBytes;
 }
 
 template <int MODE, int TN, int QM>
@@ -979,7 +1118,8 @@ bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tm_bits, cons
     auto kern = expand_gemm_kernel<MODE, TN, stages_for<MODE, TN, QM>(), QM>;
     constexpr size_t smem = smem_for<MODE, TN, QM>();
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.n_tiles, (unsigned)pl.splits);
+    const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
+    const int grid = tiles < sm_count() ? tiles : sm_count();  // persistent: one CTA per SM
     kern<<<grid, kPfThreads, smem, stream>>>(tm, tm_bits, p);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
@@ -1018,14 +1158,13 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     st = make_tmap_bits(&tm_bits, bits, d_out, pitch, q, MODE == MODE_FWD ? 128 : 64);
     if (st != BCQ_OK) return st;
 
-    BCQ_CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WsHeader), s));
     PrepParams pp;
     pp.n = n; pp.K = Kdim; pp.permute = (MODE == MODE_FWD) ? 1 : 0; pp.act_blocks = n;
     pp.ld_in = (long long)ldact; pp.ld_out = pl.ld_act;
     pp.in = reinterpret_cast<const __nv_bfloat16*>(act); pp.out = act16; pp.tok_inv_scale = tok;
     pp.alpha = alpha; pp.alpha_count = (long long)bcq_alpha_count(d_out, d_in, q, g); pp.hdr = hdr;
     long long ablocks = (pp.alpha_count + 256 * 16 - 1) / (256 * 16);
-    if (ablocks > 128) ablocks = 128;
+    if (ablocks > kMaxAlphaBlocks) ablocks = kMaxAlphaBlocks;
     if (ablocks < 1) ablocks = 1;
     prepare_kernel<<<(unsigned)(n + ablocks), 256, 0, s>>>(pp);
     bcq::count_launch();
@@ -1036,6 +1175,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.G = (int)bcq_num_groups(d_in, g);
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
+    p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
     p.alpha = alpha; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
