@@ -401,6 +401,7 @@ struct ExpandParams {
     int kb_per_split;
     int splits;
     int m_tiles, n_tiles;
+    const uint32_t* bits;
     const float* alpha;
     const float* bias;           // fwd only, may be null
     const WsHeader* hdr;         // max |alpha| per pre-pass block
@@ -427,23 +428,77 @@ struct StageLayout {
 
 // Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
 // running at the same time share activation tiles in L2).  22 warps:
-//   warp 0        TMA producer (activation tile + plane words of each stage)
+//   warp 0        TMA producer (activation tile of each stage; TMA moves about one box row per
+//                 two cycles whatever the row's size, so the plane words, 16-byte rows, stay off it)
 //   warp 1        UMMA issuer, owner of the tensor-memory allocation (two accumulators)
 //   warps 2..17   workers in two groups of eight that take alternate pipeline stages; a task is
-//                 32 weights of one row, so a group rebuilds one 128 x 64 weight tile
+//                 32 weights of one row (one plane word per plane, fetched two of the group's
+//                 stages ahead), so a group rebuilds one 128 x 64 weight tile
 //   warps 18..21  epilogue: drain one accumulator while the main loop fills the other
 constexpr int kPfWorkerWarps = 16;
 constexpr int kPfGroupWarps = 8;
 constexpr int kPfEpiWarp0 = kWorkerWarp0 + kPfWorkerWarps;  // 18
 constexpr int kPfEpiWarps = 4;
 constexpr int kPfThreads = (kPfEpiWarp0 + kPfEpiWarps) * 32;  // 704
+constexpr uint32_t kPfCtlBytes = 256;                          // barriers, TMEM handle, abort flag
+constexpr uint32_t kPfScaleBytes = 2 * 256 * 4;                // [2][TN] output scales
+constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 2048;       // per epilogue warp: 16 tokens x 32 rows fp32
+
+// The plane words and scales of one task, fetched ahead of their use.
+template <int QM>
+struct Task {
+    uint32_t w[NumWords<QM>::value];
+    float a[NumWords<QM>::value];
+    int key;  // row * G + group; -1: nothing there (expands to zeros)
+};
+
+template <int QM>
+__device__ __forceinline__ void fetch_task(Task<QM>& t, const ExpandParams& p, long long plane_words,
+                                           long long plane_alpha, int j, int kw, bool in_range, float wscale) {
+    const bool valid = in_range && (j < p.d_out) && (kw < p.pitch);
+    const int c = min((kw * 32) / p.g, p.G - 1);
+    t.key = valid ? j * p.G + c : -1;
+#pragma unroll
+    for (int i = 0; i < NumWords<QM>::value; ++i) {
+        if (i < p.q && valid) {
+            t.w[i] = __ldg(p.bits + i * plane_words + (long long)j * p.pitch + kw);
+            t.a[i] = __ldg(p.alpha + i * plane_alpha + (long long)j * p.G + c) * wscale;
+        } else {
+            t.w[i] = 0u;
+            t.a[i] = 0.0f;
+        }
+    }
+}
+
+template <int QM>
+__device__ __forceinline__ void run_task32(const Task<QM>& t, Lut& lut, int& lut_key, int q, uint32_t line,
+                                           uint32_t lx, uint32_t chunk0) {
+    if (QM == QM_GENERIC) {
+        uint32_t w8[BCQ_MAX_Q];
+        float a8[BCQ_MAX_Q];
+#pragma unroll
+        for (int i = 0; i < BCQ_MAX_Q; ++i) {
+            w8[i] = t.w[i % NumWords<QM>::value];
+            a8[i] = t.a[i % NumWords<QM>::value];
+        }
+        expand16_sum(w8, a8, q, line, lx, chunk0);
+#pragma unroll
+        for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
+        expand16_sum(w8, a8, q, line, lx, chunk0 + 2);
+    } else {
+        if (t.key != lut_key) {
+            lut = (QM == QM_LUT4) ? build_lut(t.a[0], t.a[1], t.a[2], t.a[3]) : build_lut(t.a[0], t.a[1], t.a[2], 0.0f);
+            lut_key = t.key;
+        }
+        expand32_lut<QM == QM_LUT4>(t.w[0], t.w[1], t.w[2], t.w[3], lut, line, lx, chunk0);
+    }
+}
 
 template <int MODE, int TN, int STAGES, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
-expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_bits,
-                   const ExpandParams p) {
-    using L = StageLayout<MODE, TN, QM>;
-    constexpr uint32_t kStageBytes = L::kStageBytes;
+expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParams p) {
+    constexpr uint32_t kBBytes = TN * kBlockK * 2;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
     constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
     // fp16 x fp16 -> fp32; A is MN-major for dX
     constexpr uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
@@ -465,7 +520,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 40);
     ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 44);
     ctl.device_flag = &g_timeout_flag;
-    float* out_scale = reinterpret_cast<float*>(ctl_gen + 256);  // [2][TN]: 1 / (weight scale * token scale)
+    float* out_scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [2][TN]: 1 / (weight scale * token scale)
+    const uint32_t staging_base = ctl_base + kPfCtlBytes + kPfScaleBytes;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -484,7 +540,6 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         *ctl.abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_b);
-        ptx::prefetch_tmap(&tmap_bits);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
@@ -513,21 +568,15 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             bool ok = true;
             int s = 0, in_flight = 0;
             uint32_t ph = 0;
-            const uint32_t tx = L::kBBytes + (uint32_t)p.q * L::kPlaneBytes;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int m0, t0, z, kb_begin, iters;
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
                 for (int it = 0; it < iters; ++it) {
-                    const int kb = kb_begin + it;
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const uint32_t st = smem_base + s * kStageBytes;
-                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, tx);
-                    ptx::tma_load_2d(st + kABytes, &tmap_b, kb * kBlockK, t0, ctl.full + 8 * s);
-                    if (MODE == MODE_FWD)
-                        ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, (kb >> 1) * 4, m0, 0, ctl.full + 8 * s);
-                    else
-                        ptx::tma_load_3d(st + L::kBitsOff, &tmap_bits, m0 >> 5, kb * kBlockK, 0, ctl.full + 8 * s);
+                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kBBytes);
+                    ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0,
+                                     ctl.full + 8 * s);
                     in_flight = min(in_flight + 1, STAGES);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -555,7 +604,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
                 const int acc = lt & 1;
                 const uint32_t acc_ph = (lt >> 1) & 1;
-                ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // epilogue has drained it
+                ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * TmemCols<TN>::value;
@@ -587,8 +636,19 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const int wid = warp - kWorkerWarp0;  // 0..15
         const int group = wid >> 3;           // takes the stages whose running index has this parity
         const int wl = wid & 7;
+        const long long plane_words = (long long)p.d_out * p.pitch;
         const long long plane_alpha = (long long)p.d_out * p.G;
         const float wscale = pow2f(weight_shift(p.hdr, p.q));
+
+        // fwd : task = (weight row m0 + row, 32-wide half of the stage's 64 k); the two halves of a
+        //       row sit in adjacent lanes
+        // dX  : task = (K index j = 64*kb + row, 32-wide quarter of the tile's 128 k); the four
+        //       quarters of a row sit in adjacent lanes
+        const int row = (MODE == MODE_FWD) ? wl * 16 + (lane >> 1) : wl * 8 + (lane >> 2);
+        const int part = (MODE == MODE_FWD) ? (lane & 1) : (lane & 3);
+        const uint32_t line_off = (MODE == MODE_FWD) ? row * 128 : ((part >> 1) * 8192) + row * 128;
+        const uint32_t lx = row & 7;
+        const uint32_t chunk0 = (MODE == MODE_FWD) ? part * 4 : (part & 1) * 4;
 
         Lut lut = {0u, 0u, 0u, 0u};
         int lut_key = -2;
@@ -599,75 +659,32 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
-            if (MODE == MODE_FWD) {
-                // task = (weight row, 32-wide half of the stage's 64 k); the two halves of a row sit
-                // in adjacent lanes so that their scale loads coalesce.  The scales of the group that
-                // follows are requested when the current ones are taken into use.
-                const int row = wl * 16 + (lane >> 1);
-                const int half = lane & 1;
-                const int j = m0 + row;
-                const bool valid = j < p.d_out;
-                const uint32_t line_off = row * 128, lx = row & 7, chunk0 = half * 4;
-                const uint32_t word_off = row * 16 + (half << 2);
-                const int first = (gi & 1) == group ? 0 : 1;  // first stage of this tile that is ours
-                AlphaSet<QM> cur, nxt;
-                int c_cur = min(((kb_begin + first) * kBlockK + half * 32) / p.g, p.G - 1);
-                int c_nxt = min(c_cur + max(1, 2 * kBlockK / p.g), p.G - 1);
-                load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c_cur, valid, wscale);
-                load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c_nxt, valid, wscale);
-                for (int it = 0; it < iters; ++it, ++gi) {
-                    if ((gi & 1) == group) {
-                        const int kb = kb_begin + it;
-                        const int c = min((kb * kBlockK + half * 32) / p.g, p.G - 1);
-                        if (c != c_cur) {
-                            if (c == c_nxt) cur = nxt;
-                            else load_alpha<QM>(cur, p.alpha, plane_alpha, p.G, p.q, j, c, valid, wscale);
-                            c_cur = c;
-                            c_nxt = min(c + max(1, 2 * kBlockK / p.g), p.G - 1);
-                            load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c_nxt, valid, wscale);
-                        }
-                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // plane words of the stage have landed
-                        if (!ok) break;
-                        const uint32_t st = smem_base + s * kStageBytes;
-                        expand_task32<QM>(cur, st + L::kBitsOff + word_off + ((kb & 1) << 3), L::kPlaneBytes, lut,
-                                          lut_key, p.q, st + line_off, lx, chunk0);
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                    }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+            auto fetch = [&](Task<QM>& slot, int it) {
+                const int kb = kb_begin + it;
+                if (MODE == MODE_FWD)
+                    fetch_task<QM>(slot, p, plane_words, plane_alpha, m0 + row, kb * 2 + part, it < iters, wscale);
+                else
+                    fetch_task<QM>(slot, p, plane_words, plane_alpha, kb * kBlockK + row, (m0 >> 5) + part,
+                                   it < iters, wscale);
+            };
+            // our stages of this tile are it = first, first + 2, ...; p0 / p1 hold the next two
+            const int first = ((gi & 1) == group) ? 0 : 1;
+            Task<QM> p0, p1;
+            fetch(p0, first);
+            fetch(p1, first + 2);
+            for (int it = 0; it < iters; ++it, ++gi) {
+                if ((gi & 1) == group) {
+                    const Task<QM> cur = p0;
+                    p0 = p1;
+                    fetch(p1, it + 4);
+                    ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 6);  // the UMMAs that read this slot are done
+                    if (!ok) break;
+                    run_task32<QM>(cur, lut, lut_key, p.q, smem_base + s * kStageBytes + line_off, lx, chunk0);
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
                 }
-            } else {
-                // task = (K index j = 64*kb + jl, 32-wide quarter of the tile's 128 k).  Rows change
-                // with every stage: the scales of our next stage are requested when the current ones
-                // are taken into use (two pipeline stages ahead).
-                const int jl = wl * 8 + (lane >> 2);
-                const int part = lane & 3;
-                const uint32_t line_off = ((part >> 1) * 8192) + jl * 128, lx = jl & 7, chunk0 = (part & 1) * 4;
-                const uint32_t word_off = jl * 16 + (part << 2);
-                const int c = min((m0 + part * 32) / p.g, p.G - 1);
-                const int first = (gi & 1) == group ? 0 : 1;
-                AlphaSet<QM> cur, nxt;
-                {
-                    const int j = (kb_begin + first) * kBlockK + jl;
-                    load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, j, c, (first < iters) && (j < p.d_out), wscale);
-                }
-                for (int it = 0; it < iters; ++it, ++gi) {
-                    if ((gi & 1) == group) {
-                        cur = nxt;
-                        const int jn = (kb_begin + it + 2) * kBlockK + jl;
-                        load_alpha<QM>(nxt, p.alpha, plane_alpha, p.G, p.q, jn, c, (it + 2 < iters) && (jn < p.d_out), wscale);
-                        ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);
-                        if (!ok) break;
-                        const uint32_t st = smem_base + s * kStageBytes;
-                        expand_task32<QM>(cur, st + L::kBitsOff + word_off, L::kPlaneBytes, lut, lut_key, p.q,
-                                          st + line_off, lx, chunk0);
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                    }
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
-                }
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
         }
     } else {
@@ -676,6 +693,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
         const int et = ew * 32 + lane;      // 0..127
         const float winv = pow2f(-weight_shift(p.hdr, p.q));
+        const uint32_t stg = staging_base + ew * 2048;  // this warp's staging: [16 tokens][32 rows]
+        const int esz = (p.splits > 1 || !p.out_bf16) ? 4 : 2;  // bytes per stored element
+        uint8_t* out_base = (p.splits > 1) ? reinterpret_cast<uint8_t*>(p.partial) : reinterpret_cast<uint8_t*>(p.out);
+        const long long out_ld = (p.splits > 1) ? (long long)p.Mdim : p.ldo;
+        // 16-byte stores need an aligned base and pitch
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(out_base) & 15u) == 0) && ((out_ld * esz) % 16 == 0);
         bool ok = true;
         int lt = 0;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
@@ -690,39 +713,66 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7);
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            int m = m0 + quarter * 32 + lane;
-            if (MODE == MODE_BWDX) {
-                // accumulator row r holds k = 8*(r/8) + {0,4,1,5,2,6,3,7}[r % 8]
-                const int ps = m & 7;
-                m = (m & ~7) | ((ps >> 1) + 4 * (ps & 1));
-            }
-            const bool m_ok = m < p.Mdim;
-            const float bias =
-                (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m_ok) ? __ldg(p.bias + m) : 0.0f;
+            // accumulator row `lane` of this warp's quarter is output column m0w + lrow
+            const int m0w = m0 + quarter * 32;
+            int lrow = lane;
+            if (MODE == MODE_BWDX) lrow = (lane & ~7) | (((lane & 7) >> 1) + 4 * (lane & 1));  // undo 0,4,1,5,2,6,3,7
+            const float bias = (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m0w + lrow < p.Mdim)
+                                   ? __ldg(p.bias + m0w + lrow) : 0.0f;
+            uint8_t* tile_out = out_base + ((p.splits > 1) ? (long long)z * p.n * p.Mdim * 4 : 0);
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
+            const bool full_rows = vec_ok && (m0w + 32 <= p.Mdim);
 #pragma unroll 1
             for (int col = 0; col < TN; col += 16) {
                 if (t0 + col >= p.n) break;  // uniform in the warp
                 uint32_t v[16];
                 ptx::tmem_ld_x16(t_row + (uint32_t)col, v);
                 ptx::tmem_ld_wait();
-                if (m_ok) {
+                // transpose through shared memory: staging[token][row], then 16-byte pieces of one
+                // token's 32 rows go out as coalesced vector stores
+                if (esz == 2) {
 #pragma unroll
-                    for (int cidx = 0; cidx < 16; ++cidx) {
-                        const int t = t0 + col + cidx;
-                        if (t < p.n) {
-                            const float val = __uint_as_float(v[cidx]) * scale[col + cidx];
-                            if (p.splits > 1) {
-                                p.partial[((long long)z * p.n + t) * p.Mdim + m] = val;
-                            } else if (p.out_bf16) {
-                                reinterpret_cast<__nv_bfloat16*>(p.out)[(long long)t * p.ldo + m] =
-                                    __float2bfloat16_rn(val + bias);
-                            } else {
-                                reinterpret_cast<float*>(p.out)[(long long)t * p.ldo + m] = val + bias;
+                    for (int c = 0; c < 16; ++c) {
+                        const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[c]) * scale[col + c] + bias);
+                        asm volatile("st.shared.b16 [%0], %1;" ::"r"(stg + c * 64 + lrow * 2),
+                                     "h"(*reinterpret_cast<const unsigned short*>(&h)) : "memory");
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float f = __uint_as_float(v[c]) * scale[col + c] + bias;
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + c * 128 + lrow * 4), "f"(f) : "memory");
+                    }
+                }
+                __syncwarp();
+                const int row_bytes = 32 * esz;           // one token's 32 rows
+                const int pieces = row_bytes / 16;        // 4 (bf16) or 8 (fp32) pieces per token
+                for (int pc = lane; pc < 16 * pieces; pc += 32) {
+                    const int c = pc / pieces, seg = pc - c * pieces;
+                    const int t = t0 + col + c;
+                    if (t >= p.n) continue;
+                    uint32_t r0, r1, r2, r3;
+                    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                                 : "r"(stg + c * row_bytes + seg * 16) : "memory");
+                    uint8_t* dst = tile_out + ((long long)t * out_ld + m0w) * esz + seg * 16;
+                    if (full_rows) {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(r0, r1, r2, r3);
+                    } else {
+                        const uint32_t rr[4] = {r0, r1, r2, r3};
+                        const int per = 16 / esz;  // elements in this piece
+#pragma unroll
+                        for (int e2 = 0; e2 < 8; ++e2) {
+                            if (e2 < per && m0w + seg * per + e2 < p.Mdim) {
+                                if (esz == 2)
+                                    reinterpret_cast<unsigned short*>(dst)[e2] =
+                                        (unsigned short)(rr[e2 >> 1] >> ((e2 & 1) * 16));
+                                else
+                                    reinterpret_cast<uint32_t*>(dst)[e2] = rr[e2 & 3];
                             }
                         }
                     }
                 }
+                __syncwarp();
             }
             // the accumulator (and this tile's scale row) may be reused
             ptx::tc_fence_before_sync();
@@ -1095,43 +1145,42 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
-constexpr size_t kCtlBytes = 256 + 2 * 256 * 4;     // barriers + two rows of output scales
-constexpr size_t kSmemBudget = 232448 - 1024 - kCtlBytes;  // 227 KiB minus alignment slack and the control block
+constexpr size_t kPfTailBytes = kPfCtlBytes + kPfScaleBytes + kPfStagingBytes;
+constexpr size_t kSmemBudget = 232448 - 1024 - kPfTailBytes;  // 227 KiB minus alignment slack and the tail
 
-template <int MODE, int TN, int QM>
+template <int TN>
 constexpr int stages_for() {
-    constexpr size_t per = StageLayout<MODE, TN, QM>::kStageBytes;
+    constexpr size_t per = kABytes + (size_t)TN * kBlockK * 2;
     constexpr int fit = (int)(kSmemBudget / per);
     // even, because the two worker groups alternate stages: with an even count a group meets the
     // same slots in every round and never waits on a barrier phase it has not seen complete
-    return fit >= 6 ? 6 : (fit >= 4 ? 4 : 2);
+    return fit >= 8 ? 8 : (fit >= 6 ? 6 : (fit >= 4 ? 4 : 2));
 }
 
-template <int MODE, int TN, int QM>
+template <int TN>
 constexpr size_t smem_for() {
-    return (size_t)stages_for<MODE, TN, QM>() * StageLayout<MODE, TN, QM>::kStageBytes + 1024 + kCtlBytes;
+    return (size_t)stages_for<TN>() * (kABytes + (size_t)TN * kBlockK * 2) + 1024 + kPfTailBytes;
 }
 
 template <int MODE, int TN, int QM>
-bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tm_bits, const ExpandParams& p,
-                         const ExpandPlan& pl, cudaStream_t stream) {
-    auto kern = expand_gemm_kernel<MODE, TN, stages_for<MODE, TN, QM>(), QM>;
-    constexpr size_t smem = smem_for<MODE, TN, QM>();
+bcq_status launch_expand(const CUtensorMap& tm, const ExpandParams& p, const ExpandPlan& pl, cudaStream_t stream) {
+    auto kern = expand_gemm_kernel<MODE, TN, stages_for<TN>(), QM>;
+    constexpr size_t smem = smem_for<TN>();
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();  // persistent: one CTA per SM
-    kern<<<grid, kPfThreads, smem, stream>>>(tm, tm_bits, p);
+    kern<<<grid, kPfThreads, smem, stream>>>(tm, p);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
 }
 
 template <int MODE, int TN>
-bcq_status launch_expand_q(const CUtensorMap& tm, const CUtensorMap& tm_bits, const ExpandParams& p,
-                           const ExpandPlan& pl, cudaStream_t stream) {
-    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, tm_bits, p, pl, stream);
-    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, tm_bits, p, pl, stream);
-    return launch_expand<MODE, TN, QM_GENERIC>(tm, tm_bits, p, pl, stream);
+bcq_status launch_expand_q(const CUtensorMap& tm, const ExpandParams& p, const ExpandPlan& pl,
+                           cudaStream_t stream) {
+    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, p, pl, stream);
+    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, p, pl, stream);
+    return launch_expand<MODE, TN, QM_GENERIC>(tm, p, pl, stream);
 }
 
 // act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).
@@ -1152,10 +1201,8 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     __half* act16 = reinterpret_cast<__half*>(wsb + pl.off_act);
     const int pitch = (int)bcq_pitch_words(d_in);
 
-    CUtensorMap tm, tm_bits;
+    CUtensorMap tm;
     bcq_status st = make_tmap_16bit(&tm, act16, 1, pl.ld_act, n, (size_t)pl.ld_act, pl.TN);
-    if (st != BCQ_OK) return st;
-    st = make_tmap_bits(&tm_bits, bits, d_out, pitch, q, MODE == MODE_FWD ? 128 : 64);
     if (st != BCQ_OK) return st;
 
     PrepParams pp;
@@ -1176,14 +1223,14 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
-    p.alpha = alpha; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
+    p.bits = bits; p.alpha = alpha; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
     switch (pl.TN) {
-        case 32: st = launch_expand_q<MODE, 32>(tm, tm_bits, p, pl, s); break;
-        case 64: st = launch_expand_q<MODE, 64>(tm, tm_bits, p, pl, s); break;
-        case 128: st = launch_expand_q<MODE, 128>(tm, tm_bits, p, pl, s); break;
-        default: st = launch_expand_q<MODE, 256>(tm, tm_bits, p, pl, s); break;
+        case 32: st = launch_expand_q<MODE, 32>(tm, p, pl, s); break;
+        case 64: st = launch_expand_q<MODE, 64>(tm, p, pl, s); break;
+        case 128: st = launch_expand_q<MODE, 128>(tm, p, pl, s); break;
+        default: st = launch_expand_q<MODE, 256>(tm, p, pl, s); break;
     }
     if (st != BCQ_OK) return st;
     if (pl.splits > 1) {

@@ -37,7 +37,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ct
     uint32_t spins = 0;
     while (true) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 63u) == 0u) {
+        if ((++spins & 7u) == 0u) {
             if (*ctl.abort_flag) return false;
             if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
                 *ctl.abort_flag = 1;
