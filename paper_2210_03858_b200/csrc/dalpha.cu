@@ -223,28 +223,42 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
 }
 
 // dalpha[i][j][c] (+)= scale * sum over splits and over the sub-tiles that meet group c.
-__global__ void dalpha_reduce_kernel(int d_out, int d_in, int q, int g, int G, int HN, int splits,
-                                     int n_subtiles, int slots, uint32_t plane_mask, float scale,
-                                     int accumulate, const float* __restrict__ partial,
-                                     float* __restrict__ dalpha) {
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long total = (long long)q * G * d_out;
-    if (idx >= total) return;
-    const int j = (int)(idx % d_out);
-    const long long r = idx / d_out;
-    const int c = (int)(r % G);
-    const int i = (int)(r / G);
-    if (!((plane_mask >> i) & 1u)) return;
+// Block = 32 consecutive rows j x 8 parts: part y adds every 8th partial of its output (so that
+// eight loads per output are in flight at once), then the eight sums are added in order 0..7.
+__global__ void __launch_bounds__(256)
+dalpha_reduce_kernel(int d_out, int d_in, int q, int g, int G, int HN, int splits, int n_subtiles, int slots,
+                     uint32_t plane_mask, float scale, int accumulate, const float* __restrict__ partial,
+                     float* __restrict__ dalpha) {
+    __shared__ float sums[8][32];
+    const int jx = threadIdx.x & 31, part = threadIdx.x >> 5;
+    const int jblocks = (d_out + 31) / 32;
+    const int jb = blockIdx.x % jblocks;
+    const int r = blockIdx.x / jblocks;  // (plane, group)
+    const int c = r % G;
+    const int i = r / G;
+    const int j = jb * 32 + jx;
+    if (!((plane_mask >> i) & 1u)) return;  // uniform in the block
     const int k_lo = c * g;
     const int k_hi = min(k_lo + g, d_in) - 1;
+    const int st_lo = k_lo / HN, st_n = k_hi / HN - st_lo + 1;
+    const int total = splits * st_n;
     float s = 0.0f;
-    for (int z = 0; z < splits; ++z)
-        for (int st = k_lo / HN; st <= k_hi / HN; ++st) {
+    if (j < d_out) {
+        for (int e = part; e < total; e += 8) {
+            const int z = e / st_n, st = st_lo + (e - z * st_n);
             const int slot = c - min((st * HN) / g, G - 1);
             s += __ldg(partial + ((((long long)z * n_subtiles + st) * q + i) * slots + slot) * d_out + j);
         }
-    float* dst = dalpha + ((long long)i * d_out + j) * G + c;
-    *dst = accumulate ? (*dst + scale * s) : (scale * s);
+    }
+    sums[part][jx] = s;
+    __syncthreads();
+    if (part == 0 && j < d_out) {
+        float t = 0.0f;
+#pragma unroll
+        for (int y = 0; y < 8; ++y) t += sums[y][jx];
+        float* dst = dalpha + ((long long)i * d_out + j) * G + c;
+        *dst = accumulate ? (*dst + scale * t) : (scale * t);
+    }
 }
 
 struct DalphaPlan {
@@ -354,8 +368,8 @@ extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, in
     bcq::count_launch();
     }
     BCQ_CUDA_TRY(cudaGetLastError());
-    const long long total = (long long)q * p.G * d_out;
-    dalpha_reduce_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+    const long long rblocks = (long long)q * p.G * ((d_out + 31) / 32);
+    dalpha_reduce_kernel<<<(unsigned)rblocks, 256, 0, s>>>(
         d_out, d_in, q, g, p.G, pl.HN, pl.splits, pl.n_subtiles, pl.slots, plane_mask, scale, accumulate,
         p.partial, dalpha);
     bcq::count_launch();

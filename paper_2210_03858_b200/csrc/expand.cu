@@ -318,11 +318,49 @@ struct PrepParams {
     WsHeader* hdr;
 };
 
+// One warp per token row; VPL = 16-byte vectors a lane keeps in registers between finding the
+// row's largest magnitude and writing the scaled fp16 row (VPL = 0: the row is read twice).
+// Blocks past the activation blocks scan alpha instead.
+constexpr int kPrepTokensPerBlock = 8;
+
+__device__ __forceinline__ uint32_t max_mag_bf16x8(const uint4& x, int k0, int K) {
+    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    uint32_t m = 0u;
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        if (k0 + e < K) m = max(m, (xs[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu);
+    return m;
+}
+
+__device__ __forceinline__ uint4 scale_to_fp16x8(const uint4& x, int k0, int K, float scale, int permute) {
+    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    float f[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const uint32_t b = (xs[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu;
+        f[e] = (k0 + e < K) ? __uint_as_float(b << 16) * scale : 0.0f;
+    }
+    uint4 o;
+    if (permute) {  // order 0,4,1,5,2,6,3,7 inside each run of 8
+        o.x = pack_half2(f[0], f[4]);
+        o.y = pack_half2(f[1], f[5]);
+        o.z = pack_half2(f[2], f[6]);
+        o.w = pack_half2(f[3], f[7]);
+    } else {
+        o.x = pack_half2(f[0], f[1]);
+        o.y = pack_half2(f[2], f[3]);
+        o.z = pack_half2(f[4], f[5]);
+        o.w = pack_half2(f[6], f[7]);
+    }
+    return o;
+}
+
+template <int VPL>
 __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
     __shared__ uint32_t red[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if ((int)blockIdx.x >= p.act_blocks) {
-        // ---- max |alpha|
+        // ---- max |alpha| of this block's share
         const long long nb = gridDim.x - p.act_blocks;
         uint32_t m = 0u;
         for (long long i = ((long long)blockIdx.x - p.act_blocks) * 256 + threadIdx.x; i < p.alpha_count;
@@ -340,53 +378,37 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         }
         return;
     }
-    // ---- one token row
-    const int t = blockIdx.x;
+    const int t = blockIdx.x * kPrepTokensPerBlock + warp;
+    if (t >= p.n) return;
     const uint4* src = reinterpret_cast<const uint4*>(p.in + (long long)t * p.ld_in);
     uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)t * p.ld_out);
     const int nvec = (p.K + 7) / 8;
     uint32_t m = 0u;
-    for (int v = threadIdx.x; v < nvec; v += 256) {
-        const uint4 x = __ldg(src + v);
-        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    uint4 held[VPL > 0 ? VPL : 1];
+    if (VPL > 0) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t b = (xs[e >> 1] >> ((e & 1) * 16)) & 0x7FFFu;
-            if (v * 8 + e < p.K) m = max(m, b);
+        for (int i = 0; i < VPL; ++i) {
+            const int v = lane + 32 * i;
+            held[i] = (v < nvec) ? __ldg(src + v) : make_uint4(0u, 0u, 0u, 0u);
         }
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) m = max(m, max_mag_bf16x8(held[i], (lane + 32 * i) * 8, p.K));
+    } else {
+        for (int v = lane; v < nvec; v += 32) m = max(m, max_mag_bf16x8(__ldg(src + v), v * 8, p.K));
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-    if (lane == 0) red[warp] = m;
-    __syncthreads();
-    m = 0u;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) m = max(m, red[w]);
     const int sh = shift_for(exponent_of_bits(m << 16), 14);
     const float scale = pow2f(sh);
-    if (threadIdx.x == 0) p.tok_inv_scale[t] = pow2f(-sh);
-    for (int v = threadIdx.x; v < nvec; v += 256) {
-        const uint4 x = __ldg(src + v);
-        const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
-        float f[8];
+    if (lane == 0) p.tok_inv_scale[t] = pow2f(-sh);
+    if (VPL > 0) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const uint32_t b = (xs[e >> 1] >> ((e & 1) * 16)) & 0xFFFFu;
-            f[e] = (v * 8 + e < p.K) ? __uint_as_float(b << 16) * scale : 0.0f;
+        for (int i = 0; i < VPL; ++i) {
+            const int v = lane + 32 * i;
+            if (v < nvec) dst[v] = scale_to_fp16x8(held[i], v * 8, p.K, scale, p.permute);
         }
-        uint4 o;
-        if (p.permute) {
-            o.x = pack_half2(f[0], f[4]);
-            o.y = pack_half2(f[1], f[5]);
-            o.z = pack_half2(f[2], f[6]);
-            o.w = pack_half2(f[3], f[7]);
-        } else {
-            o.x = pack_half2(f[0], f[1]);
-            o.y = pack_half2(f[2], f[3]);
-            o.z = pack_half2(f[4], f[5]);
-            o.w = pack_half2(f[6], f[7]);
-        }
-        dst[v] = o;
+    } else {
+        for (int v = lane; v < nvec; v += 32) dst[v] = scale_to_fp16x8(__ldg(src + v), v * 8, p.K, scale, p.permute);
     }
 }
 
@@ -1213,7 +1235,14 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     long long ablocks = (pp.alpha_count + 256 * 16 - 1) / (256 * 16);
     if (ablocks > kMaxAlphaBlocks) ablocks = kMaxAlphaBlocks;
     if (ablocks < 1) ablocks = 1;
-    prepare_kernel<<<(unsigned)(n + ablocks), 256, 0, s>>>(pp);
+    const int tok_blocks = ceil_div(n, kPrepTokensPerBlock);
+    pp.act_blocks = tok_blocks;
+    const unsigned pgrid = (unsigned)(tok_blocks + ablocks);
+    const int nvec = (Kdim + 7) / 8;
+    if (nvec <= 32 * 4) prepare_kernel<4><<<pgrid, 256, 0, s>>>(pp);
+    else if (nvec <= 32 * 8) prepare_kernel<8><<<pgrid, 256, 0, s>>>(pp);
+    else if (nvec <= 32 * 16) prepare_kernel<16><<<pgrid, 256, 0, s>>>(pp);
+    else prepare_kernel<0><<<pgrid, 256, 0, s>>>(pp);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
 
