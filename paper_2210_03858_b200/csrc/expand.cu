@@ -316,6 +316,19 @@ struct PrepParams {
     const float* alpha;
     long long alpha_count;
     WsHeader* hdr;
+    // Weights regrouped into the chunks one pipeline stage consumes, each chunk contiguous so that
+    // a single bulk copy brings it into shared memory (rows past d_out are written as zeros):
+    //   forward  bits_t  [m_tile][kb][q][128 rows][2 words]   the 64 k of stage kb
+    //            alpha_t [m_tile][G][q][128 rows]
+    //   dX       bits_t  [u][jb][q][64 rows][4 words]         u = 128-wide k tile, jb = 64-row block
+    //            alpha_t [jb][G][q][64 rows]
+    int mode, d_out, q, G, pitch, num_kb, amax_blocks, bits_blocks;
+    int row_tiles;   // ceil(d_out / 128)
+    int bits_cblk;   // ceil(pitch / 32): 32-word column blocks of the plane words
+    int alpha_cblk;  // ceil(G / 32)
+    const uint32_t* bits;
+    float* alpha_t;
+    uint32_t* bits_t;
 };
 
 // One warp per token row; VPL = 16-byte vectors a lane keeps in registers between finding the
@@ -359,13 +372,62 @@ template <int VPL>
 __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
     __shared__ uint32_t red[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x >= p.act_blocks + p.amax_blocks) {
+        // ---- regroup a block of 128 rows x 32 columns (plane words or scales) of one plane:
+        // coalesced reads into shared memory, then coalesced writes of the stage chunks
+        __shared__ uint32_t tile[128][33];
+        int b = (int)blockIdx.x - p.act_blocks - p.amax_blocks;
+        const bool is_alpha = b >= p.bits_blocks;
+        if (is_alpha) b -= p.bits_blocks;
+        const int cblks = is_alpha ? p.alpha_cblk : p.bits_cblk;
+        const int cb = b % cblks;
+        const int rt = (b / cblks) % p.row_tiles;
+        const int i = b / (cblks * p.row_tiles);
+        const int ncols = is_alpha ? p.G : p.pitch;
+        const uint32_t* src = is_alpha ? reinterpret_cast<const uint32_t*>(p.alpha) : p.bits;
+        src += (long long)i * p.d_out * ncols;
+#pragma unroll 4
+        for (int pass = 0; pass < 16; ++pass) {
+            const int r = pass * 8 + warp, col = cb * 32 + lane;
+            const int j = rt * 128 + r;
+            tile[r][lane] = (j < p.d_out && col < ncols) ? __ldg(src + (long long)j * ncols + col) : 0u;
+        }
+        __syncthreads();
+        const int t = threadIdx.x;
+        uint32_t* dst = is_alpha ? reinterpret_cast<uint32_t*>(p.alpha_t) : p.bits_t;
+        for (int pass = 0; pass < 16; ++pass) {
+            int r, cl;
+            if (is_alpha) { r = t & 127; cl = pass * 2 + (t >> 7); }
+            else if (p.mode == MODE_FWD) { r = t >> 1; cl = pass * 2 + (t & 1); }
+            else { r = (pass & 1) * 64 + (t >> 2); cl = (pass >> 1) * 4 + (t & 3); }
+            const int col = cb * 32 + cl;
+            if (col >= ncols) continue;
+            long long o;
+            if (p.mode == MODE_FWD) {
+                if (is_alpha) {
+                    o = (((long long)rt * p.G + col) * p.q + i) * 128 + r;
+                } else {
+                    const int kb = col >> 1;
+                    if (kb >= p.num_kb) continue;
+                    o = ((((long long)rt * p.num_kb + kb) * p.q + i) * 128 + r) * 2 + (col & 1);
+                }
+            } else {
+                const int jb = rt * 2 + (r >> 6), rr = r & 63;
+                if (jb >= p.num_kb) continue;
+                if (is_alpha) o = (((long long)jb * p.G + col) * p.q + i) * 64 + rr;
+                else o = ((((long long)(col >> 2) * p.num_kb + jb) * p.q + i) * 64 + rr) * 4 + (col & 3);
+            }
+            dst[o] = tile[r][cl];
+        }
+        return;
+    }
     if ((int)blockIdx.x >= p.act_blocks) {
-        // ---- max |alpha| of this block's share
-        const long long nb = gridDim.x - p.act_blocks;
+        // ---- max |alpha| of this block's share of the scales
+        const long long nb = p.amax_blocks;
         uint32_t m = 0u;
-        for (long long i = ((long long)blockIdx.x - p.act_blocks) * 256 + threadIdx.x; i < p.alpha_count;
-             i += nb * 256)
-            m = max(m, __float_as_uint(__ldg(p.alpha + i)) & 0x7FFFFFFFu);
+        for (long long o = ((long long)blockIdx.x - p.act_blocks) * 256 + threadIdx.x; o < p.alpha_count;
+             o += nb * 256)
+            m = max(m, __float_as_uint(__ldg(p.alpha + o)) & 0x7FFFFFFFu);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (lane == 0) red[warp] = m;
@@ -423,8 +485,14 @@ struct ExpandParams {
     int kb_per_split;
     int splits;
     int m_tiles, n_tiles;
-    const uint32_t* bits;
-    const float* alpha;
+    // pipeline geometry (chosen on the host from q and g)
+    int stages;            // even, 2..8
+    uint32_t stage_bytes;  // A tile + B tile + weight chunk, multiple of 1024
+    uint32_t bits_bytes;   // q KiB: the stage's plane words
+    uint32_t alpha_bytes;  // q * rows * 4: the scales of one group for the stage's rows
+    int alpha_parts;       // groups a stage (fwd: 64 k) or a tile (dX: 128 k) can touch: 1, 2 or 4
+    const uint32_t* bits_t;      // regrouped plane words (see PrepParams)
+    const float* alpha_t;        // regrouped scales
     const float* bias;           // fwd only, may be null
     const WsHeader* hdr;         // max |alpha| per pre-pass block
     const float* tok_inv_scale;  // [n]
@@ -450,97 +518,56 @@ struct StageLayout {
 
 // Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
 // running at the same time share activation tiles in L2).  22 warps:
-//   warp 0        TMA producer (activation tile of each stage; TMA moves about one box row per
-//                 two cycles whatever the row's size, so the plane words, 16-byte rows, stay off it)
+//   warp 0        producer: per stage one TMA tile load (activations) and two to five bulk copies
+//                 (the stage's plane words and scales, regrouped by the pre-pass into contiguous
+//                 chunks); all of them complete on the stage's `full` barrier
 //   warp 1        UMMA issuer, owner of the tensor-memory allocation (two accumulators)
-//   warps 2..17   workers in two groups of eight that take alternate pipeline stages; a task is
-//                 32 weights of one row (one plane word per plane, fetched two of the group's
-//                 stages ahead), so a group rebuilds one 128 x 64 weight tile
+//   warps 2..17   workers in two groups of eight that take alternate pipeline stages; a thread
+//                 expands 32 weights of one row per stage (one plane word per plane), so a group
+//                 rebuilds one 128 x 64 weight tile
 //   warps 18..21  epilogue: drain one accumulator while the main loop fills the other
+// One stage in shared memory: | A tile 16 KiB | B tile TN x 128 B | plane words | scales | keys |.
 constexpr int kPfWorkerWarps = 16;
 constexpr int kPfGroupWarps = 8;
 constexpr int kPfEpiWarp0 = kWorkerWarp0 + kPfWorkerWarps;  // 18
 constexpr int kPfEpiWarps = 4;
 constexpr int kPfThreads = (kPfEpiWarp0 + kPfEpiWarps) * 32;  // 704
+constexpr int kPfMaxStages = 8;
 constexpr uint32_t kPfCtlBytes = 256;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 2 * 256 * 4;                // [2][TN] output scales
-constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 2048;       // per epilogue warp: 16 tokens x 32 rows fp32
+constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 1024;       // per epilogue warp: 32 rows x 8 fp32 / 16 bf16 tokens
 
-// The plane words and scales of one task, fetched ahead of their use.
-template <int QM>
-struct Task {
-    uint32_t w[NumWords<QM>::value];
-    float a[NumWords<QM>::value];
-    int key;  // row * G + group; -1: nothing there (expands to zeros)
-};
-
-template <int QM>
-__device__ __forceinline__ void fetch_task(Task<QM>& t, const ExpandParams& p, long long plane_words,
-                                           long long plane_alpha, int j, int kw, bool in_range, float wscale) {
-    const bool valid = in_range && (j < p.d_out) && (kw < p.pitch);
-    const int c = min((kw * 32) / p.g, p.G - 1);
-    t.key = valid ? j * p.G + c : -1;
-#pragma unroll
-    for (int i = 0; i < NumWords<QM>::value; ++i) {
-        if (i < p.q && valid) {
-            t.w[i] = __ldg(p.bits + i * plane_words + (long long)j * p.pitch + kw);
-            t.a[i] = __ldg(p.alpha + i * plane_alpha + (long long)j * p.G + c) * wscale;
-        } else {
-            t.w[i] = 0u;
-            t.a[i] = 0.0f;
-        }
-    }
-}
-
-template <int QM>
-__device__ __forceinline__ void run_task32(const Task<QM>& t, Lut& lut, int& lut_key, int q, uint32_t line,
-                                           uint32_t lx, uint32_t chunk0) {
-    if (QM == QM_GENERIC) {
-        uint32_t w8[BCQ_MAX_Q];
-        float a8[BCQ_MAX_Q];
-#pragma unroll
-        for (int i = 0; i < BCQ_MAX_Q; ++i) {
-            w8[i] = t.w[i % NumWords<QM>::value];
-            a8[i] = t.a[i % NumWords<QM>::value];
-        }
-        expand16_sum(w8, a8, q, line, lx, chunk0);
-#pragma unroll
-        for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
-        expand16_sum(w8, a8, q, line, lx, chunk0 + 2);
-    } else {
-        if (t.key != lut_key) {
-            lut = (QM == QM_LUT4) ? build_lut(t.a[0], t.a[1], t.a[2], t.a[3]) : build_lut(t.a[0], t.a[1], t.a[2], 0.0f);
-            lut_key = t.key;
-        }
-        expand32_lut<QM == QM_LUT4>(t.w[0], t.w[1], t.w[2], t.w[3], lut, line, lx, chunk0);
-    }
-}
-
-template <int MODE, int TN, int STAGES, int QM>
+template <int MODE, int TN, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
 expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParams p) {
     constexpr uint32_t kBBytes = TN * kBlockK * 2;
-    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kAuxOff = kABytes + kBBytes;
     constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
+    constexpr int kRows = (MODE == MODE_FWD) ? 128 : 64;  // weight rows of one stage
+    constexpr int kUnit = (MODE == MODE_FWD) ? 2 : 4;     // plane words per row and stage
+    constexpr int NW = NumWords<QM>::value;
     // fp16 x fp16 -> fp32; A is MN-major for dX
     constexpr uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
                                 ~((1u << 7) | (1u << 10));
 
     extern __shared__ uint8_t smem_raw[];
+    const int STAGES = p.stages;
+    const uint32_t kStageBytes = p.stage_bytes;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
     const uint32_t ctl_base = smem_base + STAGES * kStageBytes;
     uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes;
+    const uint32_t keys_off = kAuxOff + p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
 
     Ctl ctl;
     ctl.full = ctl_base;
-    ctl.aready = ctl_base + 8 * STAGES;
-    ctl.empty = ctl_base + 16 * STAGES;
-    ctl.accum = ctl_base + 24 * STAGES;        // accumulator full [2]
+    ctl.aready = ctl_base + 8 * kPfMaxStages;
+    ctl.empty = ctl_base + 16 * kPfMaxStages;
+    ctl.accum = ctl_base + 24 * kPfMaxStages;   // accumulator full [2]
     const uint32_t acc_empty = ctl.accum + 16;  // accumulator drained [2]
     ctl.spare = acc_empty + 16;
-    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * STAGES + 40);
-    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * STAGES + 44);
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * kPfMaxStages + 40);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * kPfMaxStages + 44);
     ctl.device_flag = &g_timeout_flag;
     float* out_scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [2][TN]: 1 / (weight scale * token scale)
     const uint32_t staging_base = ctl_base + kPfCtlBytes + kPfScaleBytes;
@@ -585,20 +612,42 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
     };
 
     if (warp == 0) {
-        // ---------------- TMA producer
+        // ---------------- producer
         if (lane == 0) {
             bool ok = true;
             int s = 0, in_flight = 0;
             uint32_t ph = 0;
+            const uint32_t tx = kBBytes + p.bits_bytes + p.alpha_parts * p.alpha_bytes;
+            const int span = ((MODE == MODE_FWD) ? 64 : 128) / p.alpha_parts;  // k covered by one part
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int m0, t0, z, kb_begin, iters;
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
+                const int mt = m0 >> 7;
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kBBytes);
-                    ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0,
-                                     ctl.full + 8 * s);
+                    const int kb = kb_begin + it;
+                    const uint32_t stage = smem_base + s * kStageBytes;
+                    const uint32_t bar = ctl.full + 8 * s;
+                    // group index of each part; the workers compare it with the group their
+                    // lookup table was built for
+                    const int k0 = (MODE == MODE_FWD) ? kb * kBlockK : m0;
+                    int c[4];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        c[a] = (a < p.alpha_parts) ? min((k0 + a * span) / p.g, p.G - 1) : 0;
+                        ptx::st_shared_u32(stage + keys_off + 4 * a, (uint32_t)c[a]);
+                    }
+                    ptx::mbar_arrive_expect_tx(bar, tx);
+                    ptx::tma_load_2d(stage + kABytes, &tmap_b, kb * kBlockK, t0, bar);
+                    const long long chunk = (long long)mt * p.num_kb + kb;  // fwd: [m_tile][kb]; dX: [u][jb]
+                    ptx::bulk_load(stage + kAuxOff, p.bits_t + chunk * (p.bits_bytes >> 2), p.bits_bytes, bar);
+                    const long long arow = (MODE == MODE_FWD) ? mt : kb;  // alpha_t block: m_tile or jb
+#pragma unroll
+                    for (int a = 0; a < 4; ++a)
+                        if (a < p.alpha_parts)
+                            ptx::bulk_load(stage + kAuxOff + p.bits_bytes + a * p.alpha_bytes,
+                                           p.alpha_t + (arow * p.G + c[a]) * (p.alpha_bytes >> 2), p.alpha_bytes, bar);
                     in_flight = min(in_flight + 1, STAGES);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -658,8 +707,6 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         const int wid = warp - kWorkerWarp0;  // 0..15
         const int group = wid >> 3;           // takes the stages whose running index has this parity
         const int wl = wid & 7;
-        const long long plane_words = (long long)p.d_out * p.pitch;
-        const long long plane_alpha = (long long)p.d_out * p.G;
         const float wscale = pow2f(weight_shift(p.hdr, p.q));
 
         // fwd : task = (weight row m0 + row, 32-wide half of the stage's 64 k); the two halves of a
@@ -671,43 +718,67 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         const uint32_t line_off = (MODE == MODE_FWD) ? row * 128 : ((part >> 1) * 8192) + row * 128;
         const uint32_t lx = row & 7;
         const uint32_t chunk0 = (MODE == MODE_FWD) ? part * 4 : (part & 1) * 4;
+        // which of the stage's alpha parts covers this thread's 32 k
+        const int apart = (MODE == MODE_FWD) ? (p.alpha_parts == 2 ? part : 0)
+                                             : (p.alpha_parts == 4 ? part : (p.alpha_parts == 2 ? (part >> 1) : 0));
+        const uint32_t w_off = kAuxOff + (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4
+        const uint32_t a_off = kAuxOff + p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
+        const uint32_t key_off = keys_off + 4 * apart;
 
         Lut lut = {0u, 0u, 0u, 0u};
-        int lut_key = -2;
         bool ok = true;
         int s = 0, gi = 0;  // stage slot and running stage index (its parity selects the group)
         uint32_t ph = 0;
+        auto advance = [&](int k) {
+            s += k;
+            if (s >= STAGES) { s -= STAGES; ph ^= 1u; }
+        };
 
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
-            auto fetch = [&](Task<QM>& slot, int it) {
-                const int kb = kb_begin + it;
-                if (MODE == MODE_FWD)
-                    fetch_task<QM>(slot, p, plane_words, plane_alpha, m0 + row, kb * 2 + part, it < iters, wscale);
-                else
-                    fetch_task<QM>(slot, p, plane_words, plane_alpha, kb * kBlockK + row, (m0 >> 5) + part,
-                                   it < iters, wscale);
-            };
-            // our stages of this tile are it = first, first + 2, ...; p0 / p1 hold the next two
+            int lut_key = -1;  // group the table holds; rows change with the tile (and, for dX, the stage)
+            // our stages of this tile are it = first, first + 2, ...
             const int first = ((gi & 1) == group) ? 0 : 1;
-            Task<QM> p0, p1;
-            fetch(p0, first);
-            fetch(p1, first + 2);
-            for (int it = 0; it < iters; ++it, ++gi) {
-                if ((gi & 1) == group) {
-                    const Task<QM> cur = p0;
-                    p0 = p1;
-                    fetch(p1, it + 4);
-                    ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 6);  // the UMMAs that read this slot are done
-                    if (!ok) break;
-                    run_task32<QM>(cur, lut, lut_key, p.q, smem_base + s * kStageBytes + line_off, lx, chunk0);
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+            advance(min(first, iters));
+            for (int it = first; it < iters && ok; it += 2) {
+                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // the chunk has landed (and the slot was free)
+                if (!ok) break;
+                const uint32_t stage = smem_base + s * kStageBytes;
+                uint32_t w[NW];
+#pragma unroll
+                for (int i = 0; i < NW; ++i)
+                    w[i] = (i < p.q) ? ptx::ld_shared_u32(stage + w_off + i * (kRows * kUnit * 4)) : 0u;
+                if (QM == QM_GENERIC) {
+                    float a8[BCQ_MAX_Q];
+                    uint32_t w8[BCQ_MAX_Q];
+#pragma unroll
+                    for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                        a8[i] = (i < p.q) ? ptx::ld_shared_f32(stage + a_off + i * (kRows * 4)) * wscale : 0.0f;
+                        w8[i] = w[i % NW];
+                    }
+                    expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0);
+#pragma unroll
+                    for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
+                    expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0 + 2);
+                } else {
+                    const int key = (MODE == MODE_FWD) ? (int)ptx::ld_shared_u32(stage + key_off) : 0;
+                    if (MODE == MODE_BWDX || key != lut_key) {  // dX: every stage brings other rows
+                        float a[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            a[i] = (i < p.q) ? ptx::ld_shared_f32(stage + a_off + i * (kRows * 4)) * wscale : 0.0f;
+                        lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
+                        lut_key = key;
+                    }
+                    expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, stage + line_off, lx, chunk0);
                 }
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+                advance(min(2, iters - it));
             }
+            gi += iters;
         }
     } else {
         // ---------------- epilogue warps: D[row, col] -> out[t0 + col][m0 + row]
@@ -715,7 +786,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
         const int et = ew * 32 + lane;      // 0..127
         const float winv = pow2f(-weight_shift(p.hdr, p.q));
-        const uint32_t stg = staging_base + ew * 2048;  // this warp's staging: [16 tokens][32 rows]
+        const uint32_t stg = staging_base + ew * 1024;  // this warp's staging: [tokens][32 rows], 1 KiB
         const int esz = (p.splits > 1 || !p.out_bf16) ? 4 : 2;  // bytes per stored element
         uint8_t* out_base = (p.splits > 1) ? reinterpret_cast<uint8_t*>(p.partial) : reinterpret_cast<uint8_t*>(p.out);
         const long long out_ld = (p.splits > 1) ? (long long)p.Mdim : p.ldo;
@@ -744,6 +815,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
             uint8_t* tile_out = out_base + ((p.splits > 1) ? (long long)z * p.n * p.Mdim * 4 : 0);
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
             const bool full_rows = vec_ok && (m0w + 32 <= p.Mdim);
+            // one token's 32 rows are 64 (bf16) or 128 (fp32) bytes: `pieces` 16-byte vectors
+            const int pieces = 2 * esz;
+            const int toks = 1024 / (32 * esz);  // tokens per staging round: 16 (bf16) or 8 (fp32)
 #pragma unroll 1
             for (int col = 0; col < TN; col += 16) {
                 if (t0 + col >= p.n) break;  // uniform in the warp
@@ -752,49 +826,52 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                 ptx::tmem_ld_wait();
                 // transpose through shared memory: staging[token][row], then 16-byte pieces of one
                 // token's 32 rows go out as coalesced vector stores
-                if (esz == 2) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[c]) * scale[col + c] + bias);
-                        asm volatile("st.shared.b16 [%0], %1;" ::"r"(stg + c * 64 + lrow * 2),
-                                     "h"(*reinterpret_cast<const unsigned short*>(&h)) : "memory");
-                    }
-                } else {
+                for (int half = 0; half < 2; ++half) {
+                    if (esz == 2) {
+                        if (half == 1) break;
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const float f = __uint_as_float(v[c]) * scale[col + c] + bias;
-                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + c * 128 + lrow * 4), "f"(f) : "memory");
-                    }
-                }
-                __syncwarp();
-                const int row_bytes = 32 * esz;           // one token's 32 rows
-                const int pieces = row_bytes / 16;        // 4 (bf16) or 8 (fp32) pieces per token
-                for (int pc = lane; pc < 16 * pieces; pc += 32) {
-                    const int c = pc / pieces, seg = pc - c * pieces;
-                    const int t = t0 + col + c;
-                    if (t >= p.n) continue;
-                    uint32_t r0, r1, r2, r3;
-                    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                                 : "r"(stg + c * row_bytes + seg * 16) : "memory");
-                    uint8_t* dst = tile_out + ((long long)t * out_ld + m0w) * esz + seg * 16;
-                    if (full_rows) {
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(r0, r1, r2, r3);
+                        for (int c = 0; c < 16; ++c) {
+                            const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(v[c]) * scale[col + c] + bias);
+                            asm volatile("st.shared.b16 [%0], %1;" ::"r"(stg + c * 64 + lrow * 2),
+                                         "h"(*reinterpret_cast<const unsigned short*>(&h)) : "memory");
+                        }
                     } else {
-                        const uint32_t rr[4] = {r0, r1, r2, r3};
-                        const int per = 16 / esz;  // elements in this piece
 #pragma unroll
-                        for (int e2 = 0; e2 < 8; ++e2) {
-                            if (e2 < per && m0w + seg * per + e2 < p.Mdim) {
-                                if (esz == 2)
-                                    reinterpret_cast<unsigned short*>(dst)[e2] =
-                                        (unsigned short)(rr[e2 >> 1] >> ((e2 & 1) * 16));
-                                else
-                                    reinterpret_cast<uint32_t*>(dst)[e2] = rr[e2 & 3];
+                        for (int c = 0; c < 8; ++c) {
+                            const float f = __uint_as_float(v[8 * half + c]) * scale[col + 8 * half + c] + bias;
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + c * 128 + lrow * 4), "f"(f) : "memory");
+                        }
+                    }
+                    __syncwarp();
+                    const int tbase = t0 + col + ((esz == 4) ? 8 * half : 0);
+                    for (int pc = lane; pc < toks * pieces; pc += 32) {
+                        const int c = pc / pieces, seg = pc - c * pieces;
+                        const int t = tbase + c;
+                        if (t >= p.n) continue;
+                        uint32_t r0, r1, r2, r3;
+                        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                                     : "r"(stg + pc * 16) : "memory");
+                        uint8_t* dst = tile_out + ((long long)t * out_ld + m0w) * esz + seg * 16;
+                        if (full_rows) {
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(r0, r1, r2, r3);
+                        } else {
+                            const uint32_t rr[4] = {r0, r1, r2, r3};
+                            const int per = 16 / esz;  // elements in this piece
+#pragma unroll
+                            for (int e2 = 0; e2 < 8; ++e2) {
+                                if (e2 < per && m0w + seg * per + e2 < p.Mdim) {
+                                    if (esz == 2)
+                                        reinterpret_cast<unsigned short*>(dst)[e2] =
+                                            (unsigned short)(rr[e2 >> 1] >> ((e2 & 1) * 16));
+                                    else
+                                        reinterpret_cast<uint32_t*>(dst)[e2] = rr[e2 & 3];
+                                }
                             }
                         }
                     }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
             // the accumulator (and this tile's scale row) may be reused
             ptx::tc_fence_before_sync();
@@ -1109,15 +1186,25 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams 
 
 struct ExpandPlan {
     int TN, splits, kb_per_split, num_kb, m_tiles, n_tiles;
-    size_t off_tok, off_act, off_partial, total;  // workspace layout (bytes)
-    int ld_act;                                   // pitch of the fp16 activations (elements)
+    int stages, alpha_parts;
+    uint32_t stage_bytes, bits_bytes, alpha_bytes;
+    size_t smem;                                                         // dynamic shared memory of the GEMM kernel
+    size_t off_tok, off_act, off_alpha, off_bits, off_partial, total;  // workspace layout (bytes)
+    int ld_act;                                                          // pitch of the fp16 activations (elements)
 };
 
-// Tile width over tokens and the K split.  Wide token tiles amortise the expansion of a weight
-// tile over more tokens; the K split fills the SMs when the output has few tiles.
-ExpandPlan plan_expand(int Mdim, int Kdim, int n) {
+constexpr size_t kPfTailBytes = kPfCtlBytes + kPfScaleBytes + kPfStagingBytes;
+constexpr size_t kSmemBudget = 232448 - 1024 - kPfTailBytes;  // 227 KiB minus alignment slack and the tail
+
+// Tile width over tokens, the K split and the pipeline geometry.  Wide token tiles amortise the
+// expansion of a weight tile over more tokens; the K split fills the SMs when the output has few
+// tiles.
+ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     ExpandPlan pl;
     const int sms = sm_count();
+    const int Mdim = (mode == MODE_FWD) ? d_out : d_in;
+    const int Kdim = (mode == MODE_FWD) ? d_in : d_out;
+    const int G = (int)bcq_num_groups(d_in, g);
     pl.m_tiles = ceil_div(Mdim, kBlockM);
     pl.num_kb = ceil_div(Kdim, kBlockK);
     int tn;
@@ -1138,10 +1225,31 @@ ExpandPlan plan_expand(int Mdim, int Kdim, int n) {
     if (splits > 32) splits = 32;
     pl.kb_per_split = ceil_div(pl.num_kb, splits);
     pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
+
+    // one stage: A tile, B tile, the stage's plane words (q KiB), the scales of every group the
+    // stage's k range can touch, 16 bytes of group indices
+    const int rows = (mode == MODE_FWD) ? 128 : 64;
+    const int kspan = (mode == MODE_FWD) ? 64 : 128;
+    pl.alpha_parts = (g % kspan == 0) ? 1 : ((g % (kspan / 2) == 0) ? 2 : 4);
+    if (mode == MODE_FWD && pl.alpha_parts == 4) pl.alpha_parts = 2;  // g % 32 == 0 always holds
+    pl.bits_bytes = (uint32_t)q * 1024u;
+    pl.alpha_bytes = (uint32_t)(q * rows * 4);
+    pl.stage_bytes = (uint32_t)align_up(kABytes + (size_t)tn * kBlockK * 2 + pl.bits_bytes +
+                                        (size_t)pl.alpha_parts * pl.alpha_bytes + 16, 1024);
+    // even stage count, because the two worker groups alternate stages: with an even count a
+    // group meets the same slots in every round
+    int fit = (int)(kSmemBudget / pl.stage_bytes);
+    pl.stages = fit >= 8 ? 8 : (fit >= 6 ? 6 : (fit >= 4 ? 4 : 2));
+    pl.smem = (size_t)pl.stages * pl.stage_bytes + 1024 + kPfTailBytes;
+
+    const size_t chunks_bits = (size_t)pl.m_tiles * pl.num_kb;                       // [m_tile][kb] or [u][jb]
+    const size_t blocks_alpha = (size_t)((mode == MODE_FWD) ? pl.m_tiles : pl.num_kb) * G;  // [m_tile][G] or [jb][G]
     pl.ld_act = (int)align_up((size_t)Kdim, 8);
     pl.off_tok = align_up(sizeof(WsHeader), 128);
     pl.off_act = align_up(pl.off_tok + (size_t)n * sizeof(float), 128);
-    pl.off_partial = align_up(pl.off_act + (size_t)n * pl.ld_act * 2, 128);
+    pl.off_alpha = align_up(pl.off_act + (size_t)n * pl.ld_act * 2, 128);
+    pl.off_bits = align_up(pl.off_alpha + blocks_alpha * pl.alpha_bytes, 128);
+    pl.off_partial = align_up(pl.off_bits + chunks_bits * pl.bits_bytes, 128);
     pl.total = pl.off_partial + (pl.splits > 1 ? (size_t)pl.splits * n * Mdim * sizeof(float) : 0);
     return pl;
 }
@@ -1167,31 +1275,13 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
-constexpr size_t kPfTailBytes = kPfCtlBytes + kPfScaleBytes + kPfStagingBytes;
-constexpr size_t kSmemBudget = 232448 - 1024 - kPfTailBytes;  // 227 KiB minus alignment slack and the tail
-
-template <int TN>
-constexpr int stages_for() {
-    constexpr size_t per = kABytes + (size_t)TN * kBlockK * 2;
-    constexpr int fit = (int)(kSmemBudget / per);
-    // even, because the two worker groups alternate stages: with an even count a group meets the
-    // same slots in every round and never waits on a barrier phase it has not seen complete
-    return fit >= 8 ? 8 : (fit >= 6 ? 6 : (fit >= 4 ? 4 : 2));
-}
-
-template <int TN>
-constexpr size_t smem_for() {
-    return (size_t)stages_for<TN>() * (kABytes + (size_t)TN * kBlockK * 2) + 1024 + kPfTailBytes;
-}
-
 template <int MODE, int TN, int QM>
 bcq_status launch_expand(const CUtensorMap& tm, const ExpandParams& p, const ExpandPlan& pl, cudaStream_t stream) {
-    auto kern = expand_gemm_kernel<MODE, TN, stages_for<TN>(), QM>;
-    constexpr size_t smem = smem_for<TN>();
-    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    auto kern = expand_gemm_kernel<MODE, TN, QM>;
+    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();  // persistent: one CTA per SM
-    kern<<<grid, kPfThreads, smem, stream>>>(tm, p);
+    kern<<<grid, kPfThreads, pl.smem, stream>>>(tm, p);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
@@ -1212,7 +1302,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
                       int out_dtype, void* ws, size_t ws_bytes, void* stream) {
     const int Mdim = (MODE == MODE_FWD) ? d_out : d_in;
     const int Kdim = (MODE == MODE_FWD) ? d_in : d_out;
-    const ExpandPlan pl = plan_expand(Mdim, Kdim, n);
+    const ExpandPlan pl = plan_expand(MODE, d_out, d_in, q, g, n);
     if (ws == nullptr) return BCQ_ERR_NULL;
     if (ws_bytes < pl.total) return BCQ_ERR_WORKSPACE;
     if (!aligned16(ws)) return BCQ_ERR_ALIGN;
@@ -1235,9 +1325,20 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     long long ablocks = (pp.alpha_count + 256 * 16 - 1) / (256 * 16);
     if (ablocks > kMaxAlphaBlocks) ablocks = kMaxAlphaBlocks;
     if (ablocks < 1) ablocks = 1;
+    pp.mode = MODE; pp.d_out = d_out; pp.q = q; pp.G = (int)bcq_num_groups(d_in, g); pp.pitch = pitch;
+    pp.num_kb = pl.num_kb;
+    pp.amax_blocks = (int)ablocks;
+    pp.row_tiles = ceil_div(d_out, 128);
+    pp.bits_cblk = ceil_div(pitch, 32);
+    pp.alpha_cblk = ceil_div(pp.G, 32);
+    pp.bits_blocks = q * pp.row_tiles * pp.bits_cblk;
+    const int alpha_tr_blocks = q * pp.row_tiles * pp.alpha_cblk;
+    pp.bits = bits;
+    pp.alpha_t = reinterpret_cast<float*>(wsb + pl.off_alpha);
+    pp.bits_t = reinterpret_cast<uint32_t*>(wsb + pl.off_bits);
     const int tok_blocks = ceil_div(n, kPrepTokensPerBlock);
     pp.act_blocks = tok_blocks;
-    const unsigned pgrid = (unsigned)(tok_blocks + ablocks);
+    const unsigned pgrid = (unsigned)(tok_blocks + ablocks + pp.bits_blocks + alpha_tr_blocks);
     const int nvec = (Kdim + 7) / 8;
     if (nvec <= 32 * 4) prepare_kernel<4><<<pgrid, 256, 0, s>>>(pp);
     else if (nvec <= 32 * 8) prepare_kernel<8><<<pgrid, 256, 0, s>>>(pp);
@@ -1252,7 +1353,9 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
-    p.bits = bits; p.alpha = alpha; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
+    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.bits_bytes = pl.bits_bytes;
+    p.alpha_bytes = pl.alpha_bytes; p.alpha_parts = pl.alpha_parts;
+    p.bits_t = pp.bits_t; p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
     switch (pl.TN) {
@@ -1352,9 +1455,13 @@ bcq_status expand_timeout_flag(int* flag_out, int reset) {
     return BCQ_OK;
 }
 
-size_t fwd_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_expand(d_out, d_in, n).total; }
+size_t fwd_workspace_bytes(int d_out, int d_in, int q, int g, int n) {
+    return plan_expand(MODE_FWD, d_out, d_in, q, g, n).total;
+}
 size_t decode_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_decode(d_out, d_in, n).total; }
-size_t bwd_x_workspace_bytes(int d_out, int d_in, int, int, int n) { return plan_expand(d_in, d_out, n).total; }
+size_t bwd_x_workspace_bytes(int d_out, int d_in, int q, int g, int n) {
+    return plan_expand(MODE_BWDX, d_out, d_in, q, g, n).total;
+}
 }  // namespace bcq
 
 extern "C" bcq_status bcq_linear_fwd(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
