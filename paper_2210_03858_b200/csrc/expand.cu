@@ -487,7 +487,6 @@ struct ExpandParams {
     int m_tiles, n_tiles;
     // pipeline geometry (chosen on the host from q and g)
     int stages;            // even, 2..8
-    uint32_t stage_bytes;  // A tile + B tile + weight chunk, multiple of 1024
     uint32_t bits_bytes;   // q KiB: the stage's plane words
     uint32_t alpha_bytes;  // q * rows * 4: the scales of one group for the stage's rows
     int alpha_parts;       // groups a stage (fwd: 64 k) or a tile (dX: 128 k) can touch: 1, 2 or 4
@@ -526,7 +525,8 @@ struct StageLayout {
 //                 expands 32 weights of one row per stage (one plane word per plane), so a group
 //                 rebuilds one 128 x 64 weight tile
 //   warps 18..21  epilogue: drain one accumulator while the main loop fills the other
-// One stage in shared memory: | A tile 16 KiB | B tile TN x 128 B | plane words | scales | keys |.
+// Shared memory: STAGES x | A tile 16 KiB | B tile TN x 128 B |, then STAGES x | plane words | scales |
+// group indices |, then barriers, output scales and the epilogue's staging.
 constexpr int kPfWorkerWarps = 16;
 constexpr int kPfGroupWarps = 8;
 constexpr int kPfEpiWarp0 = kWorkerWarp0 + kPfWorkerWarps;  // 18
@@ -541,7 +541,7 @@ template <int MODE, int TN, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
 expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParams p) {
     constexpr uint32_t kBBytes = TN * kBlockK * 2;
-    constexpr uint32_t kAuxOff = kABytes + kBBytes;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
     constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
     constexpr int kRows = (MODE == MODE_FWD) ? 128 : 64;  // weight rows of one stage
     constexpr int kUnit = (MODE == MODE_FWD) ? 2 : 4;     // plane words per row and stage
@@ -552,12 +552,13 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
 
     extern __shared__ uint8_t smem_raw[];
     const int STAGES = p.stages;
-    const uint32_t kStageBytes = p.stage_bytes;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t ctl_base = smem_base + STAGES * kStageBytes;
-    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes;
-    const uint32_t keys_off = kAuxOff + p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
+    const uint32_t aux_base = smem_base + STAGES * kStageBytes;
+    const uint32_t keys_off = p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
+    const uint32_t kAuxBytes = keys_off + 16;
+    const uint32_t ctl_base = aux_base + STAGES * kAuxBytes;
+    uint8_t* ctl_gen = smem_gen + STAGES * (kStageBytes + kAuxBytes);
 
     Ctl ctl;
     ctl.full = ctl_base;
@@ -628,6 +629,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                     if (!ok) break;
                     const int kb = kb_begin + it;
                     const uint32_t stage = smem_base + s * kStageBytes;
+                    const uint32_t aux = aux_base + s * kAuxBytes;
                     const uint32_t bar = ctl.full + 8 * s;
                     // group index of each part; the workers compare it with the group their
                     // lookup table was built for
@@ -636,17 +638,17 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
 #pragma unroll
                     for (int a = 0; a < 4; ++a) {
                         c[a] = (a < p.alpha_parts) ? min((k0 + a * span) / p.g, p.G - 1) : 0;
-                        ptx::st_shared_u32(stage + keys_off + 4 * a, (uint32_t)c[a]);
+                        ptx::st_shared_u32(aux + keys_off + 4 * a, (uint32_t)c[a]);
                     }
                     ptx::mbar_arrive_expect_tx(bar, tx);
                     ptx::tma_load_2d(stage + kABytes, &tmap_b, kb * kBlockK, t0, bar);
                     const long long chunk = (long long)mt * p.num_kb + kb;  // fwd: [m_tile][kb]; dX: [u][jb]
-                    ptx::bulk_load(stage + kAuxOff, p.bits_t + chunk * (p.bits_bytes >> 2), p.bits_bytes, bar);
+                    ptx::bulk_load(aux, p.bits_t + chunk * (p.bits_bytes >> 2), p.bits_bytes, bar);
                     const long long arow = (MODE == MODE_FWD) ? mt : kb;  // alpha_t block: m_tile or jb
 #pragma unroll
                     for (int a = 0; a < 4; ++a)
                         if (a < p.alpha_parts)
-                            ptx::bulk_load(stage + kAuxOff + p.bits_bytes + a * p.alpha_bytes,
+                            ptx::bulk_load(aux + p.bits_bytes + a * p.alpha_bytes,
                                            p.alpha_t + (arow * p.G + c[a]) * (p.alpha_bytes >> 2), p.alpha_bytes, bar);
                     in_flight = min(in_flight + 1, STAGES);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -721,8 +723,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         // which of the stage's alpha parts covers this thread's 32 k
         const int apart = (MODE == MODE_FWD) ? (p.alpha_parts == 2 ? part : 0)
                                              : (p.alpha_parts == 4 ? part : (p.alpha_parts == 2 ? (part >> 1) : 0));
-        const uint32_t w_off = kAuxOff + (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4
-        const uint32_t a_off = kAuxOff + p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
+        const uint32_t w_off = (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4
+        const uint32_t a_off = p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
         const uint32_t key_off = keys_off + 4 * apart;
 
         Lut lut = {0u, 0u, 0u, 0u};
@@ -745,16 +747,17 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                 ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // the chunk has landed (and the slot was free)
                 if (!ok) break;
                 const uint32_t stage = smem_base + s * kStageBytes;
+                const uint32_t aux = aux_base + s * kAuxBytes;
                 uint32_t w[NW];
 #pragma unroll
                 for (int i = 0; i < NW; ++i)
-                    w[i] = (i < p.q) ? ptx::ld_shared_u32(stage + w_off + i * (kRows * kUnit * 4)) : 0u;
+                    w[i] = (i < p.q) ? ptx::ld_shared_u32(aux + w_off + i * (kRows * kUnit * 4)) : 0u;
                 if (QM == QM_GENERIC) {
                     float a8[BCQ_MAX_Q];
                     uint32_t w8[BCQ_MAX_Q];
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                        a8[i] = (i < p.q) ? ptx::ld_shared_f32(stage + a_off + i * (kRows * 4)) * wscale : 0.0f;
+                        a8[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
                         w8[i] = w[i % NW];
                     }
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0);
@@ -762,12 +765,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                     for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0 + 2);
                 } else {
-                    const int key = (MODE == MODE_FWD) ? (int)ptx::ld_shared_u32(stage + key_off) : 0;
+                    const int key = (MODE == MODE_FWD) ? (int)ptx::ld_shared_u32(aux + key_off) : 0;
                     if (MODE == MODE_BWDX || key != lut_key) {  // dX: every stage brings other rows
                         float a[4];
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            a[i] = (i < p.q) ? ptx::ld_shared_f32(stage + a_off + i * (kRows * 4)) * wscale : 0.0f;
+                            a[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
                         lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
                         lut_key = key;
                     }
@@ -1234,8 +1237,8 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     if (mode == MODE_FWD && pl.alpha_parts == 4) pl.alpha_parts = 2;  // g % 32 == 0 always holds
     pl.bits_bytes = (uint32_t)q * 1024u;
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
-    pl.stage_bytes = (uint32_t)align_up(kABytes + (size_t)tn * kBlockK * 2 + pl.bits_bytes +
-                                        (size_t)pl.alpha_parts * pl.alpha_bytes + 16, 1024);
+    pl.stage_bytes = (uint32_t)(kABytes + (size_t)tn * kBlockK * 2 + pl.bits_bytes +
+                                (size_t)pl.alpha_parts * pl.alpha_bytes + 16);
     // even stage count, because the two worker groups alternate stages: with an even count a
     // group meets the same slots in every round
     int fit = (int)(kSmemBudget / pl.stage_bytes);
@@ -1353,7 +1356,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
-    p.stages = pl.stages; p.stage_bytes = pl.stage_bytes; p.bits_bytes = pl.bits_bytes;
+    p.stages = pl.stages; p.bits_bytes = pl.bits_bytes;
     p.alpha_bytes = pl.alpha_bytes; p.alpha_parts = pl.alpha_parts;
     p.bits_t = pp.bits_t; p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
