@@ -529,9 +529,23 @@ struct StageLayout {
 // group indices |, then barriers, output scales and the epilogue's staging.
 constexpr int kPfWorkerWarps = 16;
 constexpr int kPfGroupWarps = 8;
-constexpr int kPfEpiWarp0 = kWorkerWarp0 + kPfWorkerWarps;  // 18
 constexpr int kPfEpiWarps = 4;
-constexpr int kPfThreads = (kPfEpiWarp0 + kPfEpiWarps) * 32;  // 704
+constexpr int kPfWarps = 26;
+constexpr int kPfThreads = kPfWarps * 32;  // 832
+// Warp w runs on scheduler w % 4.  The worker warps keep their scheduler's issue slots busy, and a
+// warp that issues one dependent instruction at a time (the producer, the UMMA issuer) sharing a
+// scheduler with them waits tens of cycles for each slot.  So scheduler 0 gets the control warps
+// only: 0, 12, 16 = producers, 4 = UMMA issuer, 8 = epilogue of accumulator rows 0..31; warps 20
+// and 24 leave at once.  The sixteen workers are the first sixteen warps with w % 4 != 0
+// (1..21), and warps 25, 22, 23 are the epilogue of rows 32..63, 64..95, 96..127 (a warp reaches
+// the tensor-memory lanes 32 * (w % 4) .. + 31 only).
+__device__ __forceinline__ int pf_worker_index(int warp) {
+    const int wid = warp - (warp >> 2) - 1;
+    return ((warp & 3) != 0 && wid < kPfWorkerWarps) ? wid : -1;
+}
+__device__ __forceinline__ int pf_epilogue_index(int warp) {
+    return warp == 8 ? 0 : (warp == 25 ? 1 : (warp == 22 ? 2 : (warp == 23 ? 3 : -1)));
+}
 constexpr int kPfMaxStages = 8;
 constexpr uint32_t kPfCtlBytes = 256;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 2 * 256 * 4;                // [2][TN] output scales
@@ -578,7 +592,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ctl.full + 8 * s, 1);
+            ptx::mbar_init(ctl.full + 8 * s, 3);  // one arrival per producer warp
             ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps);
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
@@ -591,7 +605,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_b);
     }
-    if (warp == 1) {
+    if (warp == 4) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
         ptx::tmem_relinquish();
     }
@@ -612,44 +626,56 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         iters = min(p.num_kb, kb_begin + p.kb_per_split) - kb_begin;
     };
 
-    if (warp == 0) {
-        // ---------------- producer
-        if (lane == 0) {
+    if (warp == 0 || warp == 12 || warp == 16) {
+        // ---------------- producers.  Issuing one copy costs a thread a few hundred cycles, so
+        // the three kinds of copies of a stage come from three warps, each walking the stages on
+        // its own: warp 0 the activation tile (TMA), warp 12 the plane words, warp 16 the scales
+        // and the group indices (lane a = part a).  Each arrives once on the stage's `full`
+        // barrier with the bytes it brings.
+        const int role = (warp == 0) ? 0 : (warp == 12 ? 1 : 2);
+        const int parts = (role == 2) ? p.alpha_parts : 1;
+        if (lane < parts) {
             bool ok = true;
             int s = 0, in_flight = 0;
             uint32_t ph = 0;
-            const uint32_t tx = kBBytes + p.bits_bytes + p.alpha_parts * p.alpha_bytes;
             const int span = ((MODE == MODE_FWD) ? 64 : 128) / p.alpha_parts;  // k covered by one part
+            const uint32_t bits_words = p.bits_bytes >> 2, alpha_words = p.alpha_bytes >> 2;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int m0, t0, z, kb_begin, iters;
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
                 const int mt = m0 >> 7;
+                // plane words: chunk [m_tile][kb] (fwd) or [u][jb] (dX), consecutive in kb
+                const uint32_t* bits_src = p.bits_t + ((long long)mt * p.num_kb + kb_begin) * bits_words;
+                // group index of this lane's part: for dX fixed by the tile; for the forward it
+                // advances with k (kept incrementally, no division in the stage loop)
+                int kpos = ((MODE == MODE_FWD) ? kb_begin * kBlockK : m0) + lane * span;
+                int c = min(kpos / p.g, p.G - 1);
+                int next_edge = (c + 1) * p.g;  // first k of the next group
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const int kb = kb_begin + it;
-                    const uint32_t stage = smem_base + s * kStageBytes;
-                    const uint32_t aux = aux_base + s * kAuxBytes;
                     const uint32_t bar = ctl.full + 8 * s;
-                    // group index of each part; the workers compare it with the group their
-                    // lookup table was built for
-                    const int k0 = (MODE == MODE_FWD) ? kb * kBlockK : m0;
-                    int c[4];
-#pragma unroll
-                    for (int a = 0; a < 4; ++a) {
-                        c[a] = (a < p.alpha_parts) ? min((k0 + a * span) / p.g, p.G - 1) : 0;
-                        ptx::st_shared_u32(aux + keys_off + 4 * a, (uint32_t)c[a]);
+                    if (role == 0) {
+                        ptx::mbar_arrive_expect_tx(bar, kBBytes);
+                        ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
+                    } else if (role == 1) {
+                        ptx::mbar_arrive_expect_tx(bar, p.bits_bytes);
+                        ptx::bulk_load(aux_base + s * kAuxBytes, bits_src, p.bits_bytes, bar);
+                        bits_src += bits_words;
+                    } else {
+                        const uint32_t aux = aux_base + s * kAuxBytes;
+                        // the workers compare the group index with the one their lookup table was built for
+                        ptx::st_shared_u32(aux + keys_off + 4 * lane, (uint32_t)c);
+                        __syncwarp((1u << parts) - 1u);
+                        if (lane == 0) ptx::mbar_arrive_expect_tx(bar, parts * p.alpha_bytes);
+                        const long long arow = (MODE == MODE_FWD) ? mt : kb_begin + it;  // alpha_t block: m_tile or jb
+                        ptx::bulk_load(aux + p.bits_bytes + lane * p.alpha_bytes,
+                                       p.alpha_t + (arow * p.G + c) * alpha_words, p.alpha_bytes, bar);
+                        if (MODE == MODE_FWD) {
+                            kpos += kBlockK;
+                            while (kpos >= next_edge && c < p.G - 1) { ++c; next_edge += p.g; }
+                        }
                     }
-                    ptx::mbar_arrive_expect_tx(bar, tx);
-                    ptx::tma_load_2d(stage + kABytes, &tmap_b, kb * kBlockK, t0, bar);
-                    const long long chunk = (long long)mt * p.num_kb + kb;  // fwd: [m_tile][kb]; dX: [u][jb]
-                    ptx::bulk_load(aux, p.bits_t + chunk * (p.bits_bytes >> 2), p.bits_bytes, bar);
-                    const long long arow = (MODE == MODE_FWD) ? mt : kb;  // alpha_t block: m_tile or jb
-#pragma unroll
-                    for (int a = 0; a < 4; ++a)
-                        if (a < p.alpha_parts)
-                            ptx::bulk_load(aux + p.bits_bytes + a * p.alpha_bytes,
-                                           p.alpha_t + (arow * p.G + c[a]) * (p.alpha_bytes >> 2), p.alpha_bytes, bar);
                     in_flight = min(in_flight + 1, STAGES);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -666,7 +692,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 4) {
         // ---------------- UMMA issuer
         if (lane == 0) {
             bool ok = true;
@@ -704,9 +730,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
                 wait_bar(ctl.spare, 0, ctl, 5);
             }
         }
-    } else if (warp < kPfEpiWarp0) {
+    } else if (pf_worker_index(warp) >= 0) {
         // ---------------- workers
-        const int wid = warp - kWorkerWarp0;  // 0..15
+        const int wid = pf_worker_index(warp);  // 0..15
         const int group = wid >> 3;           // takes the stages whose running index has this parity
         const int wl = wid & 7;
         const float wscale = pow2f(weight_shift(p.hdr, p.q));
@@ -783,9 +809,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
             }
             gi += iters;
         }
-    } else {
+    } else if (pf_epilogue_index(warp) >= 0) {
         // ---------------- epilogue warps: D[row, col] -> out[t0 + col][m0 + row]
-        const int ew = warp - kPfEpiWarp0;  // 0..3
+        const int ew = pf_epilogue_index(warp);  // 0..3
         const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
         const int et = ew * 32 + lane;      // 0..127
         const float winv = pow2f(-weight_shift(p.hdr, p.q));
@@ -885,7 +911,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 4) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }

@@ -48,6 +48,17 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ct
     }
 }
 
+// The same for a whole (converged) warp: lane 0 polls, the outcome is broadcast, and the warp
+// barrier orders the other lanes' later reads after lane 0's acquire.  Keeps the number of threads
+// polling shared-memory barriers small.
+__device__ __forceinline__ bool warp_wait_bar(uint32_t bar, uint32_t parity, const Ctl& ctl, int code) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = wait_bar(bar, parity, ctl, code) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    __syncwarp();
+    return ok != 0;
+}
+
 template <int TN>
 struct TmemCols {
     static constexpr uint32_t value = TN < 32 ? 32 : TN;

@@ -41,7 +41,10 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 // One try: the hardware may park the thread for up to `suspend_ns` while the phase is pending and
 // wakes it when the phase completes, so a waiting warp does not burn issue slots or shared-memory
 // bandwidth.  Returns whether the phase with the given parity has completed.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns = 2000u) {
+#ifndef BCQ_SUSPEND_NS
+#define BCQ_SUSPEND_NS 2000u
+#endif
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns = BCQ_SUSPEND_NS) {
     uint32_t ok;
     asm volatile(
         "{\n\t"
