@@ -269,6 +269,15 @@ def run_gpu(args):
         dist.all_reduce(ms, op=dist.ReduceOp.MAX)
     ms_per_step = float(ms.item()) / args.steps
     assert bcq.device_timeout_flag() == 0, "a kernel reported an expired wait"
+    if args.timed_only:
+        if rank == 0:
+            sampler.stop()
+            print(json.dumps({"metric": METRIC, "value": world * STEP_FLOPS / (ms_per_step * 1e-3) / 1e12, "unit": UNIT,
+                              "n_gpus": world, "steps": args.steps, "ms_per_step": ms_per_step,
+                              "gpu_launches": int(launches), "note": "timed steps only"}))
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     # ---- per-operation GPU time for the roofline: all 96 calls of one operation back to back on
     # one stream (captured as a graph so that host launch time stays out), CUDA-event timed
@@ -406,6 +415,8 @@ def main():
     ap.add_argument("--no-decode", dest="decode", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch every kernel from the host each step")
     ap.add_argument("--out-fp32", dest="out_bf16", action="store_false", help="fp32 Y and dX instead of bf16")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="warm-up and timed steps only (no per-operation, end-to-end, CPU or decode legs): the command to profile")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
