@@ -390,7 +390,17 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         for (int pass = 0; pass < 16; ++pass) {
             const int r = pass * 8 + warp, col = cb * 32 + lane;
             const int j = rt * 128 + r;
-            tile[r][lane] = (j < p.d_out && col < ncols) ? __ldg(src + (long long)j * ncols + col) : 0u;
+            uint32_t v = (j < p.d_out && col < ncols) ? __ldg(src + (long long)j * ncols + col) : 0u;
+            if (!is_alpha) {
+                // even bits of every byte to its low nibble, odd bits to the high nibble: one PRMT
+                // pair of the expansion emits weights 0,4,1,5,2,6,3,7 of a byte, so with the bits
+                // stored as 0,2,4,6,1,3,5,7 the expanded tile comes out in natural k order
+                uint32_t t = (v ^ (v >> 1)) & 0x22222222u;
+                v ^= t ^ (t << 1);
+                t = (v ^ (v >> 2)) & 0x0C0C0C0Cu;
+                v ^= t ^ (t << 2);
+            }
+            tile[r][lane] = v;
         }
         __syncthreads();
         const int t = threadIdx.x;
@@ -837,8 +847,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
             ptx::tc_fence_after_sync();
             // accumulator row `lane` of this warp's quarter is output column m0w + lrow
             const int m0w = m0 + quarter * 32;
-            int lrow = lane;
-            if (MODE == MODE_BWDX) lrow = (lane & ~7) | (((lane & 7) >> 1) + 4 * (lane & 1));  // undo 0,4,1,5,2,6,3,7
+            const int lrow = lane;
             const float bias = (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m0w + lrow < p.Mdim)
                                    ? __ldg(p.bias + m0w + lrow) : 0.0f;
             uint8_t* tile_out = out_base + ((p.splits > 1) ? (long long)z * p.n * p.Mdim * 4 : 0);
@@ -1347,7 +1356,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     if (st != BCQ_OK) return st;
 
     PrepParams pp;
-    pp.n = n; pp.K = Kdim; pp.permute = (MODE == MODE_FWD) ? 1 : 0; pp.act_blocks = n;
+    pp.n = n; pp.K = Kdim; pp.permute = 0; pp.act_blocks = n;
     pp.ld_in = (long long)ldact; pp.ld_out = pl.ld_act;
     pp.in = reinterpret_cast<const __nv_bfloat16*>(act); pp.out = act16; pp.tok_inv_scale = tok;
     pp.alpha = alpha; pp.alpha_count = (long long)bcq_alpha_count(d_out, d_in, q, g); pp.hdr = hdr;
