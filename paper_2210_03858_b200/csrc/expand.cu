@@ -508,6 +508,7 @@ struct ExpandParams {
     void* out;                   // [n][ldo]
     long long ldo;
     int out_bf16;
+    int fast_epi;                // bf16 output written by TMA stores (aligned base and pitch, no K split)
     float* partial;              // [splits][n][Mdim] when splits > 1
 };
 
@@ -558,12 +559,13 @@ __device__ __forceinline__ int pf_epilogue_index(int warp) {
 }
 constexpr int kPfMaxStages = 8;
 constexpr uint32_t kPfCtlBytes = 256;                          // barriers, TMEM handle, abort flag
-constexpr uint32_t kPfScaleBytes = 2 * 256 * 4;                // [2][TN] output scales
-constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 1024;       // per epilogue warp: 32 rows x 8 fp32 / 16 bf16 tokens
+constexpr uint32_t kPfScaleBytes = 256 * 4;                    // [TN] output scales of the tile being drained
+constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 2048;       // per epilogue warp: two 1 KiB buffers of 32 rows x 16 bf16 (8 fp32) tokens
 
 template <int MODE, int TN, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
-expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParams p) {
+expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_out,
+                   const ExpandParams p) {
     constexpr uint32_t kBBytes = TN * kBlockK * 2;
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
     constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
@@ -578,11 +580,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
     const int STAGES = p.stages;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t aux_base = smem_base + STAGES * kStageBytes;
+    const uint32_t staging_base = smem_base + STAGES * kStageBytes;  // 1 KiB aligned: the output boxes are swizzled
+    const uint32_t aux_base = staging_base + kPfStagingBytes;
     const uint32_t keys_off = p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
     const uint32_t kAuxBytes = keys_off + 16;
     const uint32_t ctl_base = aux_base + STAGES * kAuxBytes;
-    uint8_t* ctl_gen = smem_gen + STAGES * (kStageBytes + kAuxBytes);
+    uint8_t* ctl_gen = smem_gen + STAGES * (kStageBytes + kAuxBytes) + kPfStagingBytes;
 
     Ctl ctl;
     ctl.full = ctl_base;
@@ -594,8 +597,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * kPfMaxStages + 40);
     ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * kPfMaxStages + 44);
     ctl.device_flag = &g_timeout_flag;
-    float* out_scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [2][TN]: 1 / (weight scale * token scale)
-    const uint32_t staging_base = ctl_base + kPfCtlBytes + kPfScaleBytes;
+    float* scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [TN]: 1 / (weight scale * token scale)
+    const uint32_t scale_addr = ctl_base + kPfCtlBytes;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -614,6 +617,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         *ctl.abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tmap(&tmap_b);
+        if (p.fast_epi) ptx::prefetch_tmap(&tmap_out);
     }
     if (warp == 4) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
@@ -825,7 +829,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
         const int et = ew * 32 + lane;      // 0..127
         const float winv = pow2f(-weight_shift(p.hdr, p.q));
-        const uint32_t stg = staging_base + ew * 1024;  // this warp's staging: [tokens][32 rows], 1 KiB
+        const uint32_t stg = staging_base + ew * 2048;  // this warp's staging: two buffers of [tokens][32 rows], 1 KiB each
         const int esz = (p.splits > 1 || !p.out_bf16) ? 4 : 2;  // bytes per stored element
         uint8_t* out_base = (p.splits > 1) ? reinterpret_cast<uint8_t*>(p.partial) : reinterpret_cast<uint8_t*>(p.out);
         const long long out_ld = (p.splits > 1) ? (long long)p.Mdim : p.ldo;
@@ -833,12 +837,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
         const bool vec_ok = ((reinterpret_cast<uintptr_t>(out_base) & 15u) == 0) && ((out_ld * esz) % 16 == 0);
         bool ok = true;
         int lt = 0;
+        uint32_t chunks = 0;  // output boxes stored so far (fast path): selects the staging buffer
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
             const int acc = lt & 1;
             const uint32_t acc_ph = (lt >> 1) & 1;
-            float* scale = out_scale + acc * TN;
             for (int i = et; i < TN; i += kPfEpiWarps * 32)
                 scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
             asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
@@ -853,11 +857,58 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
             uint8_t* tile_out = out_base + ((p.splits > 1) ? (long long)z * p.n * p.Mdim * 4 : 0);
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
             const bool full_rows = vec_ok && (m0w + 32 <= p.Mdim);
+            if (p.fast_epi) {
+                // bf16 output through TMA stores: the accumulator is read as MMA fragments (thread
+                // t: rows g = t/4 and g + 8, token pairs 2(t%4)), scaled, packed to bf16 pairs and
+                // transposed by stmatrix into a 64-byte-swizzled [16 tokens][32 rows] box
+                const int g = lane >> 2, tq = lane & 3;
+                float b4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    b4[i] = (MODE == MODE_FWD && p.bias != nullptr && m0w + g + 8 * i < p.Mdim) ? __ldg(p.bias + m0w + g + 8 * i) : 0.0f;
+                const int tok = ((lane >> 4) << 3) + (lane & 7);  // token row this lane addresses
+                const uint32_t st_off = (uint32_t)tok * 64u;
+                const uint32_t st_sw = (uint32_t)((tok >> 1) & 3);
+                const uint32_t jb = (uint32_t)((lane >> 3) & 1);
+#pragma unroll 1
+                for (int col = 0; col < TN; col += 16) {
+                    if (t0 + col >= p.n || m0w >= p.Mdim) break;  // uniform in the warp
+                    uint32_t va[8], vb[8];
+                    ptx::tmem_ld_16x256b_x2(t_row + (uint32_t)col, va);
+                    ptx::tmem_ld_16x256b_x2(t_row + (16u << 16) + (uint32_t)col, vb);
+                    ptx::tmem_ld_wait();
+                    if (chunks >= 2) {  // the store that read this buffer two boxes ago has to be done with it
+                        if (lane == 0) ptx::bulk_wait_group_read<1>();
+                        __syncwarp();
+                    }
+                    const uint32_t buf = stg + (chunks & 1u) * 1024u;
+                    float s0x, s0y, s1x, s1y;
+                    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s0x), "=f"(s0y) : "r"(scale_addr + (col + 2 * tq) * 4) : "memory");
+                    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s1x), "=f"(s1y) : "r"(scale_addr + (col + 8 + 2 * tq) * 4) : "memory");
+                    auto pk = [](uint32_t x, uint32_t y, float sx, float sy, float b) {
+                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(x) * sx + b, __uint_as_float(y) * sy + b);
+                        return *reinterpret_cast<const uint32_t*>(&h);
+                    };
+                    const uint32_t a0 = pk(va[0], va[1], s0x, s0y, b4[0]), a1 = pk(va[2], va[3], s0x, s0y, b4[1]);
+                    const uint32_t a2 = pk(va[4], va[5], s1x, s1y, b4[0]), a3 = pk(va[6], va[7], s1x, s1y, b4[1]);
+                    const uint32_t c0 = pk(vb[0], vb[1], s0x, s0y, b4[2]), c1 = pk(vb[2], vb[3], s0x, s0y, b4[3]);
+                    const uint32_t c2 = pk(vb[4], vb[5], s1x, s1y, b4[2]), c3 = pk(vb[6], vb[7], s1x, s1y, b4[3]);
+                    ptx::stmatrix_x4_trans(buf + st_off + ((jb ^ st_sw) << 4), a0, a1, a2, a3);
+                    ptx::stmatrix_x4_trans(buf + st_off + (((jb + 2u) ^ st_sw) << 4), c0, c1, c2, c3);
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&tmap_out, m0w, t0 + col, buf);
+                        ptx::bulk_commit_group();
+                    }
+                    ++chunks;
+                }
+            }
             // one token's 32 rows are 64 (bf16) or 128 (fp32) bytes: `pieces` 16-byte vectors
             const int pieces = 2 * esz;
             const int toks = 1024 / (32 * esz);  // tokens per staging round: 16 (bf16) or 8 (fp32)
 #pragma unroll 1
-            for (int col = 0; col < TN; col += 16) {
+            for (int col = 0; col < TN && !p.fast_epi; col += 16) {
                 if (t0 + col >= p.n) break;  // uniform in the warp
                 uint32_t v[16];
                 ptx::tmem_ld_x16(t_row + (uint32_t)col, v);
@@ -916,6 +967,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const ExpandParam
             asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
             if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * acc);
         }
+        if (p.fast_epi && lane == 0) ptx::bulk_wait_group<0>();  // all output boxes written before the CTA ends
     }
 
     ptx::tc_fence_before_sync();
@@ -1314,23 +1366,24 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
 }
 
 template <int MODE, int TN, int QM>
-bcq_status launch_expand(const CUtensorMap& tm, const ExpandParams& p, const ExpandPlan& pl, cudaStream_t stream) {
+bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
+                         cudaStream_t stream) {
     auto kern = expand_gemm_kernel<MODE, TN, QM>;
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
     const int grid = tiles < sm_count() ? tiles : sm_count();  // persistent: one CTA per SM
-    kern<<<grid, kPfThreads, pl.smem, stream>>>(tm, p);
+    kern<<<grid, kPfThreads, pl.smem, stream>>>(tm, tmo, p);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     return BCQ_OK;
 }
 
 template <int MODE, int TN>
-bcq_status launch_expand_q(const CUtensorMap& tm, const ExpandParams& p, const ExpandPlan& pl,
+bcq_status launch_expand_q(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
                            cudaStream_t stream) {
-    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, p, pl, stream);
-    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, p, pl, stream);
-    return launch_expand<MODE, TN, QM_GENERIC>(tm, p, pl, stream);
+    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, tmo, p, pl, stream);
+    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, tmo, p, pl, stream);
+    return launch_expand<MODE, TN, QM_GENERIC>(tm, tmo, p, pl, stream);
 }
 
 // act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).
@@ -1396,11 +1449,18 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.bits_t = pp.bits_t; p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
+    // bf16 output with an aligned base and pitch and no K split goes out through TMA stores
+    CUtensorMap tmo = tm;
+    p.fast_epi = (p.out_bf16 && pl.splits == 1 && aligned16(out) && (ldo * 2) % 16 == 0 && ldo >= (size_t)Mdim) ? 1 : 0;
+    if (p.fast_epi) {
+        st = make_tmap_out_bf16(&tmo, out, Mdim, n, ldo);
+        if (st != BCQ_OK) return st;
+    }
     switch (pl.TN) {
-        case 32: st = launch_expand_q<MODE, 32>(tm, p, pl, s); break;
-        case 64: st = launch_expand_q<MODE, 64>(tm, p, pl, s); break;
-        case 128: st = launch_expand_q<MODE, 128>(tm, p, pl, s); break;
-        default: st = launch_expand_q<MODE, 256>(tm, p, pl, s); break;
+        case 32: st = launch_expand_q<MODE, 32>(tm, tmo, p, pl, s); break;
+        case 64: st = launch_expand_q<MODE, 64>(tm, tmo, p, pl, s); break;
+        case 128: st = launch_expand_q<MODE, 128>(tm, tmo, p, pl, s); break;
+        default: st = launch_expand_q<MODE, 256>(tm, tmo, p, pl, s); break;
     }
     if (st != BCQ_OK) return st;
     if (pl.splits > 1) {

@@ -122,6 +122,28 @@ inline bcq_status make_tmap_16bit(CUtensorMap* m, const void* base, int is_fp16,
     return BCQ_OK;
 }
 
+// bf16 output [outer][pitch_elems] with `inner` valid elements per row, written in boxes of
+// 32 x 16 elements whose 64-byte rows are 64-byte swizzled in shared memory.
+inline bcq_status make_tmap_out_bf16(CUtensorMap* m, void* base, int inner, int outer, size_t pitch_elems) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) {
+        set_last_cuda_error((int)cudaErrorNotSupported);
+        return BCQ_ERR_CUDA;
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    cuuint64_t strides[1] = {(cuuint64_t)pitch_elems * 2};
+    cuuint32_t box[2] = {32u, 16u};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_last_cuda_error((int)cudaErrorInvalidValue);
+        return BCQ_ERR_CUDA;
+    }
+    return BCQ_OK;
+}
+
 // The packed planes uint32 [q][d_out][pitch] as a 3-D tensor; box = 4 words (128 weights) x
 // box_rows x q, no swizzle; rows or words out of range read as zero.
 inline bcq_status make_tmap_bits(CUtensorMap* m, const uint32_t* bits, int d_out, int pitch_words, int q,
