@@ -558,7 +558,7 @@ __device__ __forceinline__ int pf_epilogue_index(int warp) {
     return warp == 8 ? 0 : (warp == 25 ? 1 : (warp == 22 ? 2 : (warp == 23 ? 3 : -1)));
 }
 constexpr int kPfMaxStages = 8;
-constexpr uint32_t kPfCtlBytes = 256;                          // barriers, TMEM handle, abort flag
+constexpr uint32_t kPfCtlBytes = 320;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 256 * 4;                    // [TN] output scales of the tile being drained
 constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 2048;       // per epilogue warp: two 1 KiB buffers of 32 rows x 16 bf16 (8 fp32) tokens
 
@@ -597,6 +597,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * kPfMaxStages + 40);
     ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * kPfMaxStages + 44);
     ctl.device_flag = &g_timeout_flag;
+    const uint32_t wfull = ctl_base + 256;  // + 8*s : the stage's plane words and scales have landed
     float* scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [TN]: 1 / (weight scale * token scale)
     const uint32_t scale_addr = ctl_base + kPfCtlBytes;
 
@@ -605,7 +606,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ctl.full + 8 * s, 3);  // one arrival per producer warp
+            ptx::mbar_init(ctl.full + 8 * s, 1);  // activation tile
+            ptx::mbar_init(wfull + 8 * s, 2);     // plane words, scales
             ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps);
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
@@ -668,7 +670,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const uint32_t bar = ctl.full + 8 * s;
+                    const uint32_t bar = (role == 0) ? ctl.full + 8 * s : wfull + 8 * s;
                     if (role == 0) {
                         ptx::mbar_arrive_expect_tx(bar, kBBytes);
                         ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
@@ -702,7 +704,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 for (int i = 0; i < in_flight; ++i) {
                     if (bs == 0) { bs = STAGES; bph ^= 1u; }
                     --bs;
-                    wait_bar(ctl.full + 8 * bs, bph, ctl, 2);
+                    wait_bar((role == 0) ? ctl.full + 8 * bs : wfull + 8 * bs, bph, ctl, 2);
                 }
             }
         }
@@ -784,7 +786,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const int first = ((gi & 1) == group) ? 0 : 1;
             advance(min(first, iters));
             for (int it = first; it < iters && ok; it += 2) {
-                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 6);  // the chunk has landed (and the slot was free)
+                ok = wait_bar(wfull + 8 * s, ph, ctl, 6);  // the chunk has landed (and the slot was free)
                 if (!ok) break;
                 const uint32_t stage = smem_base + s * kStageBytes;
                 const uint32_t aux = aux_base + s * kAuxBytes;
