@@ -606,9 +606,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ctl.full + 8 * s, 1);  // activation tile
             ptx::mbar_init(wfull + 8 * s, 2);     // plane words, scales
-            ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps);
+            ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps + 1);  // both operands: the worker warps and the activation tile
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -670,7 +669,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const uint32_t bar = (role == 0) ? ctl.full + 8 * s : wfull + 8 * s;
+                    const uint32_t bar = (role == 0) ? ctl.aready + 8 * s : wfull + 8 * s;
                     if (role == 0) {
                         ptx::mbar_arrive_expect_tx(bar, kBBytes);
                         ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
@@ -704,47 +703,58 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 for (int i = 0; i < in_flight; ++i) {
                     if (bs == 0) { bs = STAGES; bph ^= 1u; }
                     --bs;
-                    wait_bar((role == 0) ? ctl.full + 8 * bs : wfull + 8 * bs, bph, ctl, 2);
+                    wait_bar((role == 0) ? ctl.aready + 8 * bs : wfull + 8 * bs, bph, ctl, 2);
                 }
             }
         }
     } else if (warp == 4) {
-        // ---------------- UMMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            int s = 0, lt = 0;
-            uint32_t ph = 0;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
-                int m0, t0, z, kb_begin, iters;
-                tile_coords(tile, m0, t0, z, kb_begin, iters);
-                const int acc = lt & 1;
-                const uint32_t acc_ph = (lt >> 1) & 1;
-                ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
+        // ---------------- UMMA issuer: the whole warp walks the stages and waits on the barriers
+        // (warp-uniform control flow); one elected lane issues
+        bool ok = true;
+        int s = 0, lt = 0;
+        uint32_t ph = 0;
+        // shared-memory descriptor halves (128-byte swizzle, version 1): low = start address >> 4 and
+        // leading offset >> 4 at bit 16, high = stride offset >> 4, version at bit 14, swizzle at bit 29
+        constexpr uint32_t kHiCommon = (1024u >> 4) | (1u << 14) | (2u << 29);
+        constexpr uint32_t kAHi = kHiCommon, kBHi = kHiCommon;
+        constexpr uint32_t kALoExtra = ((MODE == MODE_FWD) ? (16u >> 4) : (8192u >> 4)) << 16;  // leading offset of A
+        constexpr uint32_t kBLoExtra = (16u >> 4) << 16;
+        constexpr uint32_t kAStep = (MODE == MODE_FWD) ? (32u >> 4) : (2048u >> 4);
+        const uint32_t a_lo0 = ((smem_base >> 4) & 0x3FFFu) | kALoExtra;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+            int m0, t0, z, kb_begin, iters;
+            tile_coords(tile, m0, t0, z, kb_begin, iters);
+            const int acc = lt & 1;
+            const uint32_t acc_ph = (lt >> 1) & 1;
+            ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + (uint32_t)acc * TmemCols<TN>::value;
+            for (int it = 0; it < iters; ++it) {
+                ok = wait_bar(ctl.aready + 8 * s, ph, ctl, 4);  // both operands of the stage are in place
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + (uint32_t)acc * TmemCols<TN>::value;
-                for (int it = 0; it < iters; ++it) {
-                    ok = wait_bar(ctl.full + 8 * s, ph, ctl, 3) && wait_bar(ctl.aready + 8 * s, ph, ctl, 4);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    const uint32_t sa = smem_base + s * kStageBytes;
-                    const uint32_t sb = sa + kABytes;
+                if (ptx::elect_one()) {
+                    // descriptors: only the start-address field changes, by 32 bytes (K-major) or
+                    // 2048 bytes (MN-major A) per UMMA
+                    const uint32_t a_lo = a_lo0 + (uint32_t)s * (kStageBytes >> 4);
+                    const uint32_t b_lo = a_lo + (kABytes >> 4) - kALoExtra + kBLoExtra;
 #pragma unroll
-                    for (int kk = 0; kk < kBlockK / 16; ++kk) {
-                        const uint64_t da = (MODE == MODE_FWD) ? ptx::make_smem_desc(sa + kk * 32, 16, 1024)
-                                                               : ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
-                        const uint64_t db = ptx::make_smem_desc(sb + kk * 32, 16, 1024);
-                        ptx::umma_bf16(d_tmem, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < kBlockK / 16; ++kk)
+                        ptx::umma_f16_halves(d_tmem, a_lo + kk * kAStep, kAHi, b_lo + kk * 2, kBHi, kIdesc,
+                                             (it > 0 || kk > 0) ? 1u : 0u);
                     ptx::umma_commit(ctl.empty + 8 * s);
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                if (ok) ptx::umma_commit(ctl.accum + 8 * acc);
+                __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
-            if (!ok) {
-                ptx::umma_commit(ctl.spare);
-                wait_bar(ctl.spare, 0, ctl, 5);
-            }
+            if (ok && ptx::elect_one()) ptx::umma_commit(ctl.accum + 8 * acc);
+            __syncwarp();
+        }
+        if (!ok) {
+            if (ptx::elect_one()) ptx::umma_commit(ctl.spare);
+            __syncwarp();
+            wait_bar(ctl.spare, 0, ctl, 5);
         }
     } else if (pf_worker_index(warp) >= 0) {
         // ---------------- workers
