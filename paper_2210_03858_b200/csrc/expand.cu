@@ -497,6 +497,8 @@ struct ExpandParams {
     int m_tiles, n_tiles;
     // pipeline geometry (chosen on the host from q and g)
     int stages;            // even, 2..8
+    int aux_slots;         // ring of plane-word / scale chunks, even, >= stages, <= 8: filled ahead of the operand slots
+    int epi_bufs;          // staging buffers per epilogue warp: 1 or 2
     uint32_t bits_bytes;   // q KiB: the stage's plane words
     uint32_t alpha_bytes;  // q * rows * 4: the scales of one group for the stage's rows
     int alpha_parts;       // groups a stage (fwd: 64 k) or a tile (dX: 128 k) can touch: 1, 2 or 4
@@ -558,9 +560,9 @@ __device__ __forceinline__ int pf_epilogue_index(int warp) {
     return warp == 8 ? 0 : (warp == 25 ? 1 : (warp == 22 ? 2 : (warp == 23 ? 3 : -1)));
 }
 constexpr int kPfMaxStages = 8;
-constexpr uint32_t kPfCtlBytes = 320;                          // barriers, TMEM handle, abort flag
+constexpr uint32_t kPfCtlBytes = 384;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 256 * 4;                    // [TN] output scales of the tile being drained
-constexpr uint32_t kPfStagingBytes = kPfEpiWarps * 2048;       // per epilogue warp: two 1 KiB buffers of 32 rows x 16 bf16 (8 fp32) tokens
+constexpr uint32_t kPfStagingBuf = kPfEpiWarps * 1024;         // per epilogue warp one 1 KiB buffer of 32 rows x 16 bf16 (8 fp32) tokens; one or two such sets
 
 template <int MODE, int TN, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
@@ -581,11 +583,13 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
     const uint32_t staging_base = smem_base + STAGES * kStageBytes;  // 1 KiB aligned: the output boxes are swizzled
-    const uint32_t aux_base = staging_base + kPfStagingBytes;
+    const int AUXS = p.aux_slots;
+    const uint32_t staging_bytes = (uint32_t)p.epi_bufs * kPfStagingBuf;
+    const uint32_t aux_base = staging_base + staging_bytes;
     const uint32_t keys_off = p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
     const uint32_t kAuxBytes = keys_off + 16;
-    const uint32_t ctl_base = aux_base + STAGES * kAuxBytes;
-    uint8_t* ctl_gen = smem_gen + STAGES * (kStageBytes + kAuxBytes) + kPfStagingBytes;
+    const uint32_t ctl_base = aux_base + AUXS * kAuxBytes;
+    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes + staging_bytes + AUXS * kAuxBytes;
 
     Ctl ctl;
     ctl.full = ctl_base;
@@ -597,7 +601,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * kPfMaxStages + 40);
     ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * kPfMaxStages + 44);
     ctl.device_flag = &g_timeout_flag;
-    const uint32_t wfull = ctl_base + 256;  // + 8*s : the stage's plane words and scales have landed
+    const uint32_t wfull = ctl_base + 256;   // + 8*a : plane words and scales of aux slot a have landed
+    const uint32_t wempty = ctl_base + 320;  // + 8*a : the worker group that used aux slot a has read it
     float* scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [TN]: 1 / (weight scale * token scale)
     const uint32_t scale_addr = ctl_base + kPfCtlBytes;
 
@@ -606,9 +611,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(wfull + 8 * s, 2);     // plane words, scales
             ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps + 1);  // both operands: the worker warps and the activation tile
             ptx::mbar_init(ctl.empty + 8 * s, 1);
+        }
+        for (int a = 0; a < AUXS; ++a) {
+            ptx::mbar_init(wfull + 8 * a, 2);  // plane words, scales
+            ptx::mbar_init(wempty + 8 * a, kPfGroupWarps);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ctl.accum + 8 * a, 1);
@@ -651,6 +659,11 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const int parts = (role == 2) ? p.alpha_parts : 1;
         if (lane < parts) {
             bool ok = true;
+            // role 0 cycles over the operand slots (freed by the UMMAs that read them), roles 1 and 2
+            // over the longer ring of weight chunks (freed by the workers as soon as they have read one)
+            const int ring = (role == 0) ? STAGES : AUXS;
+            const uint32_t free_bar = (role == 0) ? ctl.empty : wempty;
+            const uint32_t fill_bar = (role == 0) ? ctl.aready : wfull;
             int s = 0, in_flight = 0;
             uint32_t ph = 0;
             const int span = ((MODE == MODE_FWD) ? 64 : 128) / p.alpha_parts;  // k covered by one part
@@ -667,9 +680,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 int c = min(kpos / p.g, p.G - 1);
                 int next_edge = (c + 1) * p.g;  // first k of the next group
                 for (int it = 0; it < iters; ++it) {
-                    ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 1);
+                    ok = wait_bar(free_bar + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const uint32_t bar = (role == 0) ? ctl.aready + 8 * s : wfull + 8 * s;
+                    const uint32_t bar = fill_bar + 8 * s;
                     if (role == 0) {
                         ptx::mbar_arrive_expect_tx(bar, kBBytes);
                         ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
@@ -691,19 +704,19 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                             while (kpos >= next_edge && c < p.G - 1) { ++c; next_edge += p.g; }
                         }
                     }
-                    in_flight = min(in_flight + 1, STAGES);
-                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                    in_flight = min(in_flight + 1, ring);
+                    if (++s == ring) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
                 // giving up: let the copies already issued land before the CTA exits.  The last
-                // `in_flight` stages before (s, ph) were issued with the phase they had then.
+                // `in_flight` slots before (s, ph) were issued with the phase they had then.
                 int bs = s;
                 uint32_t bph = ph;
                 for (int i = 0; i < in_flight; ++i) {
-                    if (bs == 0) { bs = STAGES; bph ^= 1u; }
+                    if (bs == 0) { bs = ring; bph ^= 1u; }
                     --bs;
-                    wait_bar((role == 0) ? ctl.aready + 8 * bs : wfull + 8 * bs, bph, ctl, 2);
+                    wait_bar(fill_bar + 8 * bs, bph, ctl, 2);
                 }
             }
         }
@@ -781,11 +794,13 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
         Lut lut = {0u, 0u, 0u, 0u};
         bool ok = true;
-        int s = 0, gi = 0;  // stage slot and running stage index (its parity selects the group)
-        uint32_t ph = 0;
+        int s = 0, as = 0, gi = 0;  // operand slot, aux slot, running stage index (its parity selects the group)
+        uint32_t ph = 0, aph = 0;
         auto advance = [&](int k) {
             s += k;
             if (s >= STAGES) { s -= STAGES; ph ^= 1u; }
+            as += k;
+            if (as >= AUXS) { as -= AUXS; aph ^= 1u; }
         };
 
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
@@ -796,14 +811,21 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const int first = ((gi & 1) == group) ? 0 : 1;
             advance(min(first, iters));
             for (int it = first; it < iters && ok; it += 2) {
-                ok = wait_bar(wfull + 8 * s, ph, ctl, 6);  // the chunk has landed (and the slot was free)
+                ok = wait_bar(wfull + 8 * as, aph, ctl, 6);  // the chunk has landed
                 if (!ok) break;
                 const uint32_t stage = smem_base + s * kStageBytes;
-                const uint32_t aux = aux_base + s * kAuxBytes;
+                const uint32_t aux = aux_base + as * kAuxBytes;
                 uint32_t w[NW];
 #pragma unroll
                 for (int i = 0; i < NW; ++i)
                     w[i] = (i < p.q) ? ptx::ld_shared_u32(aux + w_off + i * (kRows * kUnit * 4)) : 0u;
+                // everything this warp needs from the chunk is in registers: hand the aux slot back,
+                // then wait until the UMMAs that read the operand slot's previous contents are done
+                auto release_and_acquire = [&]() {
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(wempty + 8 * as);
+                    return wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9);
+                };
                 if (QM == QM_GENERIC) {
                     float a8[BCQ_MAX_Q];
                     uint32_t w8[BCQ_MAX_Q];
@@ -812,6 +834,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                         a8[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
                         w8[i] = w[i % NW];
                     }
+                    ok = release_and_acquire();
+                    if (!ok) break;
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0);
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
@@ -826,6 +850,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                         lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
                         lut_key = key;
                     }
+                    ok = release_and_acquire();
+                    if (!ok) break;
                     expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, stage + line_off, lx, chunk0);
                 }
                 ptx::fence_proxy_async_smem();
@@ -841,7 +867,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const int quarter = warp & 3;       // TMEM lanes 32 * quarter .. + 31
         const int et = ew * 32 + lane;      // 0..127
         const float winv = pow2f(-weight_shift(p.hdr, p.q));
-        const uint32_t stg = staging_base + ew * 2048;  // this warp's staging: two buffers of [tokens][32 rows], 1 KiB each
+        const uint32_t stg = staging_base + ew * 1024;  // this warp's staging: [tokens][32 rows], 1 KiB (a second one kPfStagingBuf further)
         const int esz = (p.splits > 1 || !p.out_bf16) ? 4 : 2;  // bytes per stored element
         uint8_t* out_base = (p.splits > 1) ? reinterpret_cast<uint8_t*>(p.partial) : reinterpret_cast<uint8_t*>(p.out);
         const long long out_ld = (p.splits > 1) ? (long long)p.Mdim : p.ldo;
@@ -889,11 +915,14 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     ptx::tmem_ld_16x256b_x2(t_row + (uint32_t)col, va);
                     ptx::tmem_ld_16x256b_x2(t_row + (16u << 16) + (uint32_t)col, vb);
                     ptx::tmem_ld_wait();
-                    if (chunks >= 2) {  // the store that read this buffer two boxes ago has to be done with it
-                        if (lane == 0) ptx::bulk_wait_group_read<1>();
-                        __syncwarp();
+                    // the store that last read this buffer has to be done with it
+                    if (p.epi_bufs == 2) {
+                        if (chunks >= 2 && lane == 0) ptx::bulk_wait_group_read<1>();
+                    } else {
+                        if (chunks >= 1 && lane == 0) ptx::bulk_wait_group_read<0>();
                     }
-                    const uint32_t buf = stg + (chunks & 1u) * 1024u;
+                    __syncwarp();
+                    const uint32_t buf = stg + ((p.epi_bufs == 2) ? (chunks & 1u) * kPfStagingBuf : 0u);
                     float s0x, s0y, s1x, s1y;
                     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s0x), "=f"(s0y) : "r"(scale_addr + (col + 2 * tq) * 4) : "memory");
                     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s1x), "=f"(s1y) : "r"(scale_addr + (col + 8 + 2 * tq) * 4) : "memory");
@@ -1288,15 +1317,15 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams 
 
 struct ExpandPlan {
     int TN, splits, kb_per_split, num_kb, m_tiles, n_tiles;
-    int stages, alpha_parts;
-    uint32_t stage_bytes, bits_bytes, alpha_bytes;
+    int stages, aux_slots, epi_bufs, alpha_parts;
+    uint32_t bits_bytes, alpha_bytes;
     size_t smem;                                                         // dynamic shared memory of the GEMM kernel
     size_t off_tok, off_act, off_alpha, off_bits, off_partial, total;  // workspace layout (bytes)
     int ld_act;                                                          // pitch of the fp16 activations (elements)
 };
 
-constexpr size_t kPfTailBytes = kPfCtlBytes + kPfScaleBytes + kPfStagingBytes;
-constexpr size_t kSmemBudget = 232448 - 1024 - kPfTailBytes;  // 227 KiB minus alignment slack and the tail
+constexpr size_t kSmemLimit = 232448;                                   // 227 KiB per CTA
+constexpr size_t kPfFixedBytes = 1024 + kPfCtlBytes + kPfScaleBytes;   // alignment slack, barriers, output scales
 
 // Tile width over tokens, the K split and the pipeline geometry.  Wide token tiles amortise the
 // expansion of a weight tile over more tokens; the K split fills the SMs when the output has few
@@ -1336,13 +1365,29 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     if (mode == MODE_FWD && pl.alpha_parts == 4) pl.alpha_parts = 2;  // g % 32 == 0 always holds
     pl.bits_bytes = (uint32_t)q * 1024u;
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
-    pl.stage_bytes = (uint32_t)(kABytes + (size_t)tn * kBlockK * 2 + pl.bits_bytes +
-                                (size_t)pl.alpha_parts * pl.alpha_bytes + 16);
-    // even stage count, because the two worker groups alternate stages: with an even count a
-    // group meets the same slots in every round
-    int fit = (int)(kSmemBudget / pl.stage_bytes);
-    pl.stages = fit >= 8 ? 8 : (fit >= 6 ? 6 : (fit >= 4 ? 4 : 2));
-    pl.smem = (size_t)pl.stages * pl.stage_bytes + 1024 + kPfTailBytes;
+    const size_t ab_bytes = kABytes + (size_t)tn * kBlockK * 2;
+    const size_t aux_bytes = pl.bits_bytes + (size_t)pl.alpha_parts * pl.alpha_bytes + 16;
+    auto smem_of = [&](int stages, int aux_slots, int epi_bufs) {
+        return stages * ab_bytes + aux_slots * aux_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
+    };
+    // operand slots first (even count, because the two worker groups alternate stages: with an
+    // even count a group meets the same slots in every round), then a longer ring of weight
+    // chunks and a second staging buffer for the epilogue as far as they fit
+    pl.stages = 2;
+    for (int st = 8; st >= 2; st -= 2)
+        if (smem_of(st, st, 1) <= kSmemLimit) { pl.stages = st; break; }
+    pl.aux_slots = pl.stages;
+    pl.epi_bufs = 1;
+    const int tries[5][2] = {{4, 2}, {2, 2}, {4, 1}, {2, 1}, {0, 2}};
+    for (int t = 0; t < 5; ++t) {
+        const int ax = pl.stages + tries[t][0];
+        if (ax <= kPfMaxStages && smem_of(pl.stages, ax, tries[t][1]) <= kSmemLimit) {
+            pl.aux_slots = ax;
+            pl.epi_bufs = tries[t][1];
+            break;
+        }
+    }
+    pl.smem = smem_of(pl.stages, pl.aux_slots, pl.epi_bufs);
 
     const size_t chunks_bits = (size_t)pl.m_tiles * pl.num_kb;                       // [m_tile][kb] or [u][jb]
     const size_t blocks_alpha = (size_t)((mode == MODE_FWD) ? pl.m_tiles : pl.num_kb) * G;  // [m_tile][G] or [jb][G]
@@ -1456,7 +1501,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
-    p.stages = pl.stages; p.bits_bytes = pl.bits_bytes;
+    p.stages = pl.stages; p.aux_slots = pl.aux_slots; p.epi_bufs = pl.epi_bufs; p.bits_bytes = pl.bits_bytes;
     p.alpha_bytes = pl.alpha_bytes; p.alpha_parts = pl.alpha_parts;
     p.bits_t = pp.bits_t; p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
