@@ -529,36 +529,31 @@ struct StageLayout {
 };
 
 // Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
-// running at the same time share activation tiles in L2).  22 warps:
-//   warp 0        producer: per stage one TMA tile load (activations) and two to five bulk copies
-//                 (the stage's plane words and scales, regrouped by the pre-pass into contiguous
-//                 chunks); all of them complete on the stage's `full` barrier
-//   warp 1        UMMA issuer, owner of the tensor-memory allocation (two accumulators)
-//   warps 2..17   workers in two groups of eight that take alternate pipeline stages; a thread
-//                 expands 32 weights of one row per stage (one plane word per plane), so a group
-//                 rebuilds one 128 x 64 weight tile
-//   warps 18..21  epilogue: drain one accumulator while the main loop fills the other
-// Shared memory: STAGES x | A tile 16 KiB | B tile TN x 128 B |, then STAGES x | plane words | scales |
-// group indices |, then barriers, output scales and the epilogue's staging.
-constexpr int kPfWorkerWarps = 16;
+// running at the same time share activation tiles in L2).  32 warps:
+//   warps 0..23   workers in three groups of eight; group g takes the pipeline stages whose running
+//                 index is g mod 3.  A thread expands 32 weights of one row per stage (one plane
+//                 word per plane), so a group rebuilds one 128 x 64 weight tile.  The expansion is
+//                 a chain of dependent shifts, masks and PRMTs, so it is the number of warps in
+//                 flight, not the issue rate, that bounds it
+//   warp 24       UMMA issuer, owner of the tensor-memory allocation (two accumulators)
+//   warps 25..27  producers: the activation tile of a stage (TMA), its plane words and its scales
+//                 (bulk copies of the chunks the pre-pass regrouped)
+//   warps 28..31  epilogue: drain one accumulator while the main loop fills the other (warp w
+//                 reaches the tensor-memory lanes 32 * (w % 4) .. + 31)
+// Shared memory: STAGES x | A tile 16 KiB | B tile TN x 128 B |, the epilogue's staging, AUXS x
+// | plane words | scales | group indices |, then barriers and output scales.
+constexpr int kPfGroups = 3;
 constexpr int kPfGroupWarps = 8;
+constexpr int kPfWorkerWarps = kPfGroups * kPfGroupWarps;  // 24
+constexpr int kPfMmaWarp = kPfWorkerWarps;                 // 24
+constexpr int kPfProdWarp0 = kPfMmaWarp + 1;               // 25, 26, 27
+constexpr int kPfEpiWarp0 = kPfProdWarp0 + 3;              // 28
 constexpr int kPfEpiWarps = 4;
-constexpr int kPfWarps = 26;
-constexpr int kPfThreads = kPfWarps * 32;  // 832
-// Warp w runs on scheduler w % 4.  The worker warps keep their scheduler's issue slots busy, and a
-// warp that issues one dependent instruction at a time (the producer, the UMMA issuer) sharing a
-// scheduler with them waits tens of cycles for each slot.  So scheduler 0 gets the control warps
-// only: 0, 12, 16 = producers, 4 = UMMA issuer, 8 = epilogue of accumulator rows 0..31; warps 20
-// and 24 leave at once.  The sixteen workers are the first sixteen warps with w % 4 != 0
-// (1..21), and warps 25, 22, 23 are the epilogue of rows 32..63, 64..95, 96..127 (a warp reaches
-// the tensor-memory lanes 32 * (w % 4) .. + 31 only).
-__device__ __forceinline__ int pf_worker_index(int warp) {
-    const int wid = warp - (warp >> 2) - 1;
-    return ((warp & 3) != 0 && wid < kPfWorkerWarps) ? wid : -1;
-}
-__device__ __forceinline__ int pf_epilogue_index(int warp) {
-    return warp == 8 ? 0 : (warp == 25 ? 1 : (warp == 22 ? 2 : (warp == 23 ? 3 : -1)));
-}
+constexpr int kPfWarps = kPfEpiWarp0 + kPfEpiWarps;        // 32
+constexpr int kPfThreads = kPfWarps * 32;                  // 1024
+static_assert(kPfEpiWarp0 % 4 == 0, "epilogue warp e must sit on tensor-memory lane quarter e");
+__device__ __forceinline__ int pf_worker_index(int warp) { return warp < kPfWorkerWarps ? warp : -1; }
+__device__ __forceinline__ int pf_epilogue_index(int warp) { return warp >= kPfEpiWarp0 ? warp - kPfEpiWarp0 : -1; }
 constexpr int kPfMaxStages = 8;
 constexpr uint32_t kPfCtlBytes = 384;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 256 * 4;                    // [TN] output scales of the tile being drained
@@ -628,7 +623,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         ptx::prefetch_tmap(&tmap_b);
         if (p.fast_epi) ptx::prefetch_tmap(&tmap_out);
     }
-    if (warp == 4) {
+    if (warp == kPfMmaWarp) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
         ptx::tmem_relinquish();
     }
@@ -649,13 +644,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         iters = min(p.num_kb, kb_begin + p.kb_per_split) - kb_begin;
     };
 
-    if (warp == 0 || warp == 12 || warp == 16) {
+    if (warp >= kPfProdWarp0 && warp < kPfEpiWarp0) {
         // ---------------- producers.  Issuing one copy costs a thread a few hundred cycles, so
         // the three kinds of copies of a stage come from three warps, each walking the stages on
-        // its own: warp 0 the activation tile (TMA), warp 12 the plane words, warp 16 the scales
-        // and the group indices (lane a = part a).  Each arrives once on the stage's `full`
-        // barrier with the bytes it brings.
-        const int role = (warp == 0) ? 0 : (warp == 12 ? 1 : 2);
+        // its own: the activation tile (TMA), the plane words, the scales with the group indices
+        // (lane a = part a).  Each arrives on the barrier of what it fills with the bytes it brings.
+        const int role = warp - kPfProdWarp0;
         const int parts = (role == 2) ? p.alpha_parts : 1;
         if (lane < parts) {
             bool ok = true;
@@ -720,7 +714,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 }
             }
         }
-    } else if (warp == 4) {
+    } else if (warp == kPfMmaWarp) {
         // ---------------- UMMA issuer: the whole warp walks the stages and waits on the barriers
         // (warp-uniform control flow); one elected lane issues
         bool ok = true;
@@ -771,8 +765,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         }
     } else if (pf_worker_index(warp) >= 0) {
         // ---------------- workers
-        const int wid = pf_worker_index(warp);  // 0..15
-        const int group = wid >> 3;           // takes the stages whose running index has this parity
+        const int wid = pf_worker_index(warp);  // 0..23
+        const int group = wid >> 3;           // takes the stages whose running index is `group` mod kPfGroups
         const int wl = wid & 7;
         const float wscale = pow2f(weight_shift(p.hdr, p.q));
 
@@ -794,7 +788,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
         Lut lut = {0u, 0u, 0u, 0u};
         bool ok = true;
-        int s = 0, as = 0, gi = 0;  // operand slot, aux slot, running stage index (its parity selects the group)
+        int s = 0, as = 0, gi = 0;  // operand slot, aux slot, running stage index mod kPfGroups
         uint32_t ph = 0, aph = 0;
         auto advance = [&](int k) {
             s += k;
@@ -807,10 +801,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
             int lut_key = -1;  // group the table holds; rows change with the tile (and, for dX, the stage)
-            // our stages of this tile are it = first, first + 2, ...
-            const int first = ((gi & 1) == group) ? 0 : 1;
+            // our stages of this tile are it = first, first + kPfGroups, ...
+            const int first = (group - gi + kPfGroups) % kPfGroups;
             advance(min(first, iters));
-            for (int it = first; it < iters && ok; it += 2) {
+            for (int it = first; it < iters && ok; it += kPfGroups) {
                 ok = wait_bar(wfull + 8 * as, aph, ctl, 6);  // the chunk has landed
                 if (!ok) break;
                 const uint32_t stage = smem_base + s * kStageBytes;
@@ -857,9 +851,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                advance(min(2, iters - it));
+                advance(min(kPfGroups, iters - it));
             }
-            gi += iters;
+            gi = (gi + iters) % kPfGroups;
         }
     } else if (pf_epilogue_index(warp) >= 0) {
         // ---------------- epilogue warps: D[row, col] -> out[t0 + col][m0 + row]
@@ -1013,7 +1007,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == kPfMmaWarp) {
         ptx::tc_fence_after_sync();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -1370,15 +1364,16 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     auto smem_of = [&](int stages, int aux_slots, int epi_bufs) {
         return stages * ab_bytes + aux_slots * aux_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
     };
-    // operand slots first (even count, because the two worker groups alternate stages: with an
-    // even count a group meets the same slots in every round), then a longer ring of weight
-    // chunks and a second staging buffer for the epilogue as far as they fit
-    pl.stages = 2;
-    for (int st = 8; st >= 2; st -= 2)
+    // operand slots first (a multiple of the number of worker groups, which take stages in turn:
+    // then a group meets the same slots in every round and never waits on a barrier phase it has
+    // not seen complete), then a longer ring of weight chunks and a second staging buffer for the
+    // epilogue as far as they fit
+    pl.stages = kPfGroups;
+    for (int st = (kPfMaxStages / kPfGroups) * kPfGroups; st >= kPfGroups; st -= kPfGroups)
         if (smem_of(st, st, 1) <= kSmemLimit) { pl.stages = st; break; }
     pl.aux_slots = pl.stages;
     pl.epi_bufs = 1;
-    const int tries[5][2] = {{4, 2}, {2, 2}, {4, 1}, {2, 1}, {0, 2}};
+    const int tries[5][2] = {{2 * kPfGroups, 2}, {kPfGroups, 2}, {2 * kPfGroups, 1}, {kPfGroups, 1}, {0, 2}};
     for (int t = 0; t < 5; ++t) {
         const int ax = pl.stages + tries[t][0];
         if (ax <= kPfMaxStages && smem_of(pl.stages, ax, tries[t][1]) <= kSmemLimit) {
