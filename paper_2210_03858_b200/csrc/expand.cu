@@ -581,8 +581,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     const int AUXS = p.aux_slots;
     const uint32_t staging_bytes = (uint32_t)p.epi_bufs * kPfStagingBuf;
     const uint32_t aux_base = staging_base + staging_bytes;
-    const uint32_t keys_off = p.bits_bytes + p.alpha_parts * p.alpha_bytes;  // 4 ints
-    const uint32_t kAuxBytes = keys_off + 16;
+    const uint32_t kAuxBytes = p.bits_bytes + p.alpha_parts * p.alpha_bytes;
     const uint32_t ctl_base = aux_base + AUXS * kAuxBytes;
     uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes + staging_bytes + AUXS * kAuxBytes;
 
@@ -610,7 +609,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
         for (int a = 0; a < AUXS; ++a) {
-            ptx::mbar_init(wfull + 8 * a, 2);  // plane words, scales
+            ptx::mbar_init(wfull + 8 * a, 1 + p.alpha_parts);  // plane words; each part of the scales
             ptx::mbar_init(wempty + 8 * a, kPfGroupWarps);
         }
         for (int a = 0; a < 2; ++a) {
@@ -673,6 +672,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 int kpos = ((MODE == MODE_FWD) ? kb_begin * kBlockK : m0) + lane * span;
                 int c = min(kpos / p.g, p.G - 1);
                 int next_edge = (c + 1) * p.g;  // first k of the next group
+                int hist0 = -1, hist1 = -1, hist2 = -1;  // group index of this part 3, 2, 1 stages ago
+                static_assert(kPfGroups == 3, "the history covers three stages");
+                // scales: block [m_tile][G] (fwd) or [jb][G] (dX) of alpha_words each
+                const float* alpha_src = p.alpha_t + (long long)((MODE == MODE_FWD) ? mt : kb_begin) * p.G * alpha_words;
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(free_bar + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
@@ -685,17 +688,24 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                         ptx::bulk_load(aux_base + s * kAuxBytes, bits_src, p.bits_bytes, bar);
                         bits_src += bits_words;
                     } else {
-                        const uint32_t aux = aux_base + s * kAuxBytes;
-                        // the workers compare the group index with the one their lookup table was built for
-                        ptx::st_shared_u32(aux + keys_off + 4 * lane, (uint32_t)c);
-                        __syncwarp((1u << parts) - 1u);
-                        if (lane == 0) ptx::mbar_arrive_expect_tx(bar, parts * p.alpha_bytes);
-                        const long long arow = (MODE == MODE_FWD) ? mt : kb_begin + it;  // alpha_t block: m_tile or jb
-                        ptx::bulk_load(aux + p.bits_bytes + lane * p.alpha_bytes,
-                                       p.alpha_t + (arow * p.G + c) * alpha_words, p.alpha_bytes, bar);
+                        // a worker rebuilds its lookup table when the group index differs from the
+                        // one of its previous stage (kPfGroups stages back) and at its first stage
+                        // of a tile; for dX every stage brings other rows.  Only then does it read
+                        // the scales, so only then are they copied.
+                        const bool need = (MODE == MODE_BWDX) || (QM == QM_GENERIC) || (c != hist0);  // q > 4: no table, read every stage
+                        hist0 = hist1; hist1 = hist2; hist2 = c;
+                        if (need) {
+                            ptx::mbar_arrive_expect_tx(bar, p.alpha_bytes);
+                            ptx::bulk_load(aux_base + s * kAuxBytes + p.bits_bytes + lane * p.alpha_bytes,
+                                           alpha_src + (long long)c * alpha_words, p.alpha_bytes, bar);
+                        } else {
+                            ptx::mbar_arrive(bar);
+                        }
                         if (MODE == MODE_FWD) {
                             kpos += kBlockK;
                             while (kpos >= next_edge && c < p.G - 1) { ++c; next_edge += p.g; }
+                        } else {
+                            alpha_src += (long long)p.G * alpha_words;  // next block of 64 rows
                         }
                     }
                     in_flight = min(in_flight + 1, ring);
@@ -784,7 +794,6 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                                              : (p.alpha_parts == 4 ? part : (p.alpha_parts == 2 ? (part >> 1) : 0));
         const uint32_t w_off = (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4
         const uint32_t a_off = p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
-        const uint32_t key_off = keys_off + 4 * apart;
 
         Lut lut = {0u, 0u, 0u, 0u};
         bool ok = true;
@@ -801,6 +810,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
             int lut_key = -1;  // group the table holds; rows change with the tile (and, for dX, the stage)
+            // group index of this thread's 32 k at its stages (forward), kept incrementally
+            int kpos = (kb_begin + ((group - gi + kPfGroups) % kPfGroups)) * kBlockK + apart * 32;
+            int cw = min(kpos / p.g, p.G - 1);
+            int next_edge = (cw + 1) * p.g;
             // our stages of this tile are it = first, first + kPfGroups, ...
             const int first = (group - gi + kPfGroups) % kPfGroups;
             advance(min(first, iters));
@@ -835,7 +848,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0 + 2);
                 } else {
-                    const int key = (MODE == MODE_FWD) ? (int)ptx::ld_shared_u32(aux + key_off) : 0;
+                    const int key = cw;
                     if (MODE == MODE_BWDX || key != lut_key) {  // dX: every stage brings other rows
                         float a[4];
 #pragma unroll
@@ -852,6 +865,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
                 advance(min(kPfGroups, iters - it));
+                if (MODE == MODE_FWD) {
+                    kpos += kPfGroups * kBlockK;
+                    while (kpos >= next_edge && cw < p.G - 1) { ++cw; next_edge += p.g; }
+                }
             }
             gi = (gi + iters) % kPfGroups;
         }
@@ -1360,7 +1377,7 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     pl.bits_bytes = (uint32_t)q * 1024u;
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
     const size_t ab_bytes = kABytes + (size_t)tn * kBlockK * 2;
-    const size_t aux_bytes = pl.bits_bytes + (size_t)pl.alpha_parts * pl.alpha_bytes + 16;
+    const size_t aux_bytes = pl.bits_bytes + (size_t)pl.alpha_parts * pl.alpha_bytes;
     auto smem_of = [&](int stages, int aux_slots, int epi_bufs) {
         return stages * ab_bytes + aux_slots * aux_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
     };
