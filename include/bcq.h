@@ -115,7 +115,10 @@ bcq_status bcq_dequantize(int d_out, int d_in, int q, int g, const uint32_t* bit
  *   X    in : bf16 [n][ldx]
  *   bias in : float [d_out] or NULL (the frozen bias of the layer)
  *   Y    out: y_dtype [n][ldy], ldy >= d_out
- *   ws      : scratch of bcq_workspace_bytes(BCQ_OP_FWD, ...) bytes, 16-byte aligned (NULL if 0)
+ *   ws      : scratch of bcq_workspace_bytes(BCQ_OP_FWD, ...) bytes, 16-byte aligned (NULL if 0);
+ *             it holds an fp16 copy of X and a regrouped copy of the planes and scales, so it
+ *             is about 2*n*d_in + bcq_bits_bytes() + 4*bcq_alpha_count() bytes (the same,
+ *             with dY and d_out, for bcq_linear_bwd_x)
  * Arithmetic: the scaled weight sum_i alpha_i b_i is formed in fp32 and rounded once to fp16;
  * the bf16 activations are converted exactly to fp16 after a per-token power-of-two scaling
  * that is undone on output; products are accumulated in fp32 in the tensor core.  The same

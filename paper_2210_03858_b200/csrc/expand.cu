@@ -22,10 +22,11 @@
 //     gradients leave the fp16 range.  The same pre-pass finds max|alpha|, from which a power of
 //     two for the weights is derived.  Decode (<= 16 tokens) has no pre-pass: every CTA converts
 //     the X slice it needs itself and scales per (token, K-slice) and per weight row.
-//   * within every aligned run of 8 consecutive k the tile stores k in the order
-//     0,4,1,5,2,6,3,7 (that is what one PRMT pair produces).  For the forward the pre-pass writes
-//     the activations in the same order; for dX, where k indexes accumulator rows, the epilogue
-//     maps rows back.
+//   * one PRMT pair emits the weights of a byte of a plane word in the order 0,4,1,5,2,6,3,7.
+//     For the forward and dX the pre-pass, which regroups the plane words anyway, stores the bits
+//     of every byte as 0,2,4,6,1,3,5,7, so that the expanded tile is in natural k order.  Decode
+//     has no pre-pass: there the tile keeps the PRMT order and the workers write the activations
+//     in the same order.
 #include <mutex>
 
 #include "gemm_common.cuh"
