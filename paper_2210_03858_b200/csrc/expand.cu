@@ -644,6 +644,44 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         iters = min(p.num_kb, kb_begin + p.kb_per_split) - kb_begin;
     };
 
+    // bf16 output through TMA stores, 16 tokens x 32 rows at a time: the accumulator is read as MMA
+    // fragments (thread t: rows g = t/4 and g + 8 of each half of the warp's 32 lanes, token pairs
+    // 2(t%4)), scaled, packed to bf16 pairs and transposed by stmatrix into a 64-byte-swizzled
+    // [16 tokens][32 rows] box at `buf`, which one lane then hands to the TMA.  s0*, s1* are the
+    // output scales of the thread's tokens in the first and second group of eight.
+    auto store_box = [&](uint32_t t_row, int col, uint32_t buf, float s0x, float s0y, float s1x, float s1y,
+                         const float (&b4)[4], int x, int y) {
+        const int tok = ((lane >> 4) << 3) + (lane & 7);  // token row this lane addresses
+        const uint32_t st_off = (uint32_t)tok * 64u;
+        const uint32_t st_sw = (uint32_t)((tok >> 1) & 3);
+        const uint32_t jb = (uint32_t)((lane >> 3) & 1);
+        uint32_t va[8], vb[8];
+        ptx::tmem_ld_16x256b_x2(t_row + (uint32_t)col, va);
+        ptx::tmem_ld_16x256b_x2(t_row + (16u << 16) + (uint32_t)col, vb);
+        ptx::tmem_ld_wait();
+        auto pk = [](uint32_t u, uint32_t v, float sx, float sy, float b) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(u) * sx + b, __uint_as_float(v) * sy + b);
+            return *reinterpret_cast<const uint32_t*>(&h);
+        };
+        const uint32_t a0 = pk(va[0], va[1], s0x, s0y, b4[0]), a1 = pk(va[2], va[3], s0x, s0y, b4[1]);
+        const uint32_t a2 = pk(va[4], va[5], s1x, s1y, b4[0]), a3 = pk(va[6], va[7], s1x, s1y, b4[1]);
+        const uint32_t c0 = pk(vb[0], vb[1], s0x, s0y, b4[2]), c1 = pk(vb[2], vb[3], s0x, s0y, b4[3]);
+        const uint32_t c2 = pk(vb[4], vb[5], s1x, s1y, b4[2]), c3 = pk(vb[6], vb[7], s1x, s1y, b4[3]);
+        ptx::stmatrix_x4_trans(buf + st_off + ((jb ^ st_sw) << 4), a0, a1, a2, a3);
+        ptx::stmatrix_x4_trans(buf + st_off + (((jb + 2u) ^ st_sw) << 4), c0, c1, c2, c3);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+            ptx::tma_store_2d(&tmap_out, x, y, buf);
+            ptx::bulk_commit_group();
+        }
+    };
+    // On the last tile of a CTA the worker warps have nothing left to expand, so they share its
+    // epilogue: of the seven warps on a tensor-memory lane quarter (one epilogue warp, six workers)
+    // warp h takes the boxes h, h + 7, ...
+    constexpr int kPfHelpers = 1 + kPfWorkerWarps / 4;  // 7
+    auto is_last_tile = [&](int tile) { return tile + (int)gridDim.x >= num_tiles; };
+
     if (warp >= kPfProdWarp0 && warp < kPfEpiWarp0) {
         // ---------------- producers.  Issuing one copy costs a thread a few hundred cycles, so
         // the three kinds of copies of a stage come from three warps, each walking the stages on
@@ -873,6 +911,44 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             }
             gi = (gi + iters) % kPfGroups;
         }
+        if (p.fast_epi && ok && (int)blockIdx.x < num_tiles) {
+            // share the epilogue of this CTA's last tile.  Its operand slots are free once the
+            // accumulator is complete, so each warp stages its boxes in 1 KiB of the first slots.
+            const int lt = (num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x;
+            const int tile = (int)blockIdx.x + lt * (int)gridDim.x;
+            int m0, t0, z, kb_begin, iters;
+            tile_coords(tile, m0, t0, z, kb_begin, iters);
+            const int acc = lt & 1;
+            ok = wait_bar(ctl.accum + 8 * acc, (uint32_t)(lt >> 1) & 1u, ctl, 10);
+            if (ok) {
+                ptx::tc_fence_after_sync();
+                const int quarter = warp & 3, helper = 1 + (warp >> 2);  // 1..6
+                const int m0w = m0 + quarter * 32;
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
+                const uint32_t buf = smem_base + (uint32_t)warp * 1024u;
+                const float winv = 1.0f / wscale;  // a power of two
+                const int g = lane >> 2, tq = lane & 3;
+                float b4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    b4[i] = (MODE == MODE_FWD && p.bias != nullptr && m0w + g + 8 * i < p.Mdim) ? __ldg(p.bias + m0w + g + 8 * i) : 0.0f;
+                bool stored = false;
+#pragma unroll 1
+                for (int col = 16 * helper; col < TN; col += 16 * kPfHelpers) {
+                    if (t0 + col >= p.n || m0w >= p.Mdim) break;  // uniform in the warp
+                    if (stored && lane == 0) ptx::bulk_wait_group_read<0>();
+                    __syncwarp();
+                    const int ta = t0 + col + 2 * tq, tb = ta + 8;
+                    const float s0x = (ta < p.n) ? winv * __ldg(p.tok_inv_scale + ta) : 0.0f;
+                    const float s0y = (ta + 1 < p.n) ? winv * __ldg(p.tok_inv_scale + ta + 1) : 0.0f;
+                    const float s1x = (tb < p.n) ? winv * __ldg(p.tok_inv_scale + tb) : 0.0f;
+                    const float s1y = (tb + 1 < p.n) ? winv * __ldg(p.tok_inv_scale + tb + 1) : 0.0f;
+                    store_box(t_row, col, buf, s0x, s0y, s1x, s1y, b4, m0w, t0 + col);
+                    stored = true;
+                }
+                if (lane == 0) ptx::bulk_wait_group<0>();
+            }
+        }
     } else if (pf_epilogue_index(warp) >= 0) {
         // ---------------- epilogue warps: D[row, col] -> out[t0 + col][m0 + row]
         const int ew = pf_epilogue_index(warp);  // 0..3
@@ -908,25 +984,15 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
             const bool full_rows = vec_ok && (m0w + 32 <= p.Mdim);
             if (p.fast_epi) {
-                // bf16 output through TMA stores: the accumulator is read as MMA fragments (thread
-                // t: rows g = t/4 and g + 8, token pairs 2(t%4)), scaled, packed to bf16 pairs and
-                // transposed by stmatrix into a 64-byte-swizzled [16 tokens][32 rows] box
                 const int g = lane >> 2, tq = lane & 3;
                 float b4[4];
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     b4[i] = (MODE == MODE_FWD && p.bias != nullptr && m0w + g + 8 * i < p.Mdim) ? __ldg(p.bias + m0w + g + 8 * i) : 0.0f;
-                const int tok = ((lane >> 4) << 3) + (lane & 7);  // token row this lane addresses
-                const uint32_t st_off = (uint32_t)tok * 64u;
-                const uint32_t st_sw = (uint32_t)((tok >> 1) & 3);
-                const uint32_t jb = (uint32_t)((lane >> 3) & 1);
+                const int cstep = is_last_tile(tile) ? 16 * kPfHelpers : 16;  // the workers take the other boxes
 #pragma unroll 1
-                for (int col = 0; col < TN; col += 16) {
+                for (int col = 0; col < TN; col += cstep) {
                     if (t0 + col >= p.n || m0w >= p.Mdim) break;  // uniform in the warp
-                    uint32_t va[8], vb[8];
-                    ptx::tmem_ld_16x256b_x2(t_row + (uint32_t)col, va);
-                    ptx::tmem_ld_16x256b_x2(t_row + (16u << 16) + (uint32_t)col, vb);
-                    ptx::tmem_ld_wait();
                     // the store that last read this buffer has to be done with it
                     if (p.epi_bufs == 2) {
                         if (chunks >= 2 && lane == 0) ptx::bulk_wait_group_read<1>();
@@ -938,22 +1004,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     float s0x, s0y, s1x, s1y;
                     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s0x), "=f"(s0y) : "r"(scale_addr + (col + 2 * tq) * 4) : "memory");
                     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(s1x), "=f"(s1y) : "r"(scale_addr + (col + 8 + 2 * tq) * 4) : "memory");
-                    auto pk = [](uint32_t x, uint32_t y, float sx, float sy, float b) {
-                        const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(x) * sx + b, __uint_as_float(y) * sy + b);
-                        return *reinterpret_cast<const uint32_t*>(&h);
-                    };
-                    const uint32_t a0 = pk(va[0], va[1], s0x, s0y, b4[0]), a1 = pk(va[2], va[3], s0x, s0y, b4[1]);
-                    const uint32_t a2 = pk(va[4], va[5], s1x, s1y, b4[0]), a3 = pk(va[6], va[7], s1x, s1y, b4[1]);
-                    const uint32_t c0 = pk(vb[0], vb[1], s0x, s0y, b4[2]), c1 = pk(vb[2], vb[3], s0x, s0y, b4[3]);
-                    const uint32_t c2 = pk(vb[4], vb[5], s1x, s1y, b4[2]), c3 = pk(vb[6], vb[7], s1x, s1y, b4[3]);
-                    ptx::stmatrix_x4_trans(buf + st_off + ((jb ^ st_sw) << 4), a0, a1, a2, a3);
-                    ptx::stmatrix_x4_trans(buf + st_off + (((jb + 2u) ^ st_sw) << 4), c0, c1, c2, c3);
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        ptx::tma_store_2d(&tmap_out, m0w, t0 + col, buf);
-                        ptx::bulk_commit_group();
-                    }
+                    store_box(t_row, col, buf, s0x, s0y, s1x, s1y, b4, m0w, t0 + col);
                     ++chunks;
                 }
             }
