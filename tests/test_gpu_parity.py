@@ -162,7 +162,10 @@ def test_fwd_matches_oracle(n, d_in, d_out, q, g):
     bias = synth.bias(d_out, (100, n, 0))
     Yb = bcq.linear_fwd(Xd, bd, ad, d_in, g, bias=torch.from_numpy(bias).cuda(),
                         out_dtype=torch.bfloat16)
+    Yb2 = bcq.linear_fwd(Xd, bd, ad, d_in, g, bias=torch.from_numpy(bias).cuda(),
+                         out_dtype=torch.bfloat16)
     refb = ref + bias.astype(np.float64)
+    assert torch.equal(Yb, Yb2), "two bf16 runs differ"
     assert rel_err(Yb.float().cpu().numpy(), refb) <= TOL + 2.0 ** -8
 
 
@@ -177,6 +180,8 @@ def test_bwd_x_matches_oracle(n, d_in, d_out, q, g):
     assert torch.equal(dX, dX2)
     assert rel_err(dX.cpu().numpy(), ref) <= TOL
     dXb = bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=torch.bfloat16)
+    dXb2 = bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=torch.bfloat16)
+    assert torch.equal(dXb, dXb2), "two bf16 runs differ"
     assert rel_err(dXb.float().cpu().numpy(), ref) <= TOL + 2.0 ** -8
 
 
