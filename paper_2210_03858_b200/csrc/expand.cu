@@ -309,7 +309,7 @@ __device__ __forceinline__ int weight_shift(const WsHeader* hdr, int q) {
 }
 
 struct PrepParams {
-    int n, K, permute, act_blocks;
+    int n, K, act_blocks;
     long long ld_in, ld_out;
     const __nv_bfloat16* in;
     __half* out;
@@ -346,7 +346,7 @@ __device__ __forceinline__ uint32_t max_mag_bf16x8(const uint4& x, int k0, int K
     return m;
 }
 
-__device__ __forceinline__ uint4 scale_to_fp16x8(const uint4& x, int k0, int K, float scale, int permute) {
+__device__ __forceinline__ uint4 scale_to_fp16x8(const uint4& x, int k0, int K, float scale) {
     const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
     float f[8];
 #pragma unroll
@@ -355,17 +355,10 @@ __device__ __forceinline__ uint4 scale_to_fp16x8(const uint4& x, int k0, int K, 
         f[e] = (k0 + e < K) ? __uint_as_float(b << 16) * scale : 0.0f;
     }
     uint4 o;
-    if (permute) {  // order 0,4,1,5,2,6,3,7 inside each run of 8
-        o.x = pack_half2(f[0], f[4]);
-        o.y = pack_half2(f[1], f[5]);
-        o.z = pack_half2(f[2], f[6]);
-        o.w = pack_half2(f[3], f[7]);
-    } else {
-        o.x = pack_half2(f[0], f[1]);
-        o.y = pack_half2(f[2], f[3]);
-        o.z = pack_half2(f[4], f[5]);
-        o.w = pack_half2(f[6], f[7]);
-    }
+    o.x = pack_half2(f[0], f[1]);
+    o.y = pack_half2(f[2], f[3]);
+    o.z = pack_half2(f[4], f[5]);
+    o.w = pack_half2(f[6], f[7]);
     return o;
 }
 
@@ -387,11 +380,17 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         const int ncols = is_alpha ? p.G : p.pitch;
         const uint32_t* src = is_alpha ? reinterpret_cast<const uint32_t*>(p.alpha) : p.bits;
         src += (long long)i * p.d_out * ncols;
-#pragma unroll 4
+        // all sixteen loads of a thread in flight at once: the block's time is one memory latency
+        uint32_t held[16];
+        const int col_l = cb * 32 + lane;
+#pragma unroll
         for (int pass = 0; pass < 16; ++pass) {
-            const int r = pass * 8 + warp, col = cb * 32 + lane;
-            const int j = rt * 128 + r;
-            uint32_t v = (j < p.d_out && col < ncols) ? __ldg(src + (long long)j * ncols + col) : 0u;
+            const int j = rt * 128 + pass * 8 + warp;
+            held[pass] = (j < p.d_out && col_l < ncols) ? __ldg(src + (long long)j * ncols + col_l) : 0u;
+        }
+#pragma unroll
+        for (int pass = 0; pass < 16; ++pass) {
+            uint32_t v = held[pass];
             if (!is_alpha) {
                 // even bits of every byte to its low nibble, odd bits to the high nibble: one PRMT
                 // pair of the expansion emits weights 0,4,1,5,2,6,3,7 of a byte, so with the bits
@@ -401,11 +400,12 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
                 t = (v ^ (v >> 2)) & 0x0C0C0C0Cu;
                 v ^= t ^ (t << 2);
             }
-            tile[r][lane] = v;
+            tile[pass * 8 + warp][lane] = v;
         }
         __syncthreads();
         const int t = threadIdx.x;
         uint32_t* dst = is_alpha ? reinterpret_cast<uint32_t*>(p.alpha_t) : p.bits_t;
+#pragma unroll 4
         for (int pass = 0; pass < 16; ++pass) {
             int r, cl;
             if (is_alpha) { r = t & 127; cl = pass * 2 + (t >> 7); }
@@ -478,10 +478,10 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
 #pragma unroll
         for (int i = 0; i < VPL; ++i) {
             const int v = lane + 32 * i;
-            if (v < nvec) dst[v] = scale_to_fp16x8(held[i], v * 8, p.K, scale, p.permute);
+            if (v < nvec) dst[v] = scale_to_fp16x8(held[i], v * 8, p.K, scale);
         }
     } else {
-        for (int v = lane; v < nvec; v += 32) dst[v] = scale_to_fp16x8(__ldg(src + v), v * 8, p.K, scale, p.permute);
+        for (int v = lane; v < nvec; v += 32) dst[v] = scale_to_fp16x8(__ldg(src + v), v * 8, p.K, scale);
     }
 }
 
@@ -497,8 +497,8 @@ struct ExpandParams {
     int splits;
     int m_tiles, n_tiles;
     // pipeline geometry (chosen on the host from q and g)
-    int stages;            // even, 2..8
-    int aux_slots;         // ring of plane-word / scale chunks, even, >= stages, <= 8: filled ahead of the operand slots
+    int stages;            // operand slots: a multiple of the number of worker groups, <= 8
+    int aux_slots;         // ring of plane-word / scale chunks: same rule, >= stages; filled ahead of the operand slots
     int epi_bufs;          // staging buffers per epilogue warp: 1 or 2
     uint32_t bits_bytes;   // q KiB: the stage's plane words
     uint32_t alpha_bytes;  // q * rows * 4: the scales of one group for the stage's rows
@@ -1530,7 +1530,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     if (st != BCQ_OK) return st;
 
     PrepParams pp;
-    pp.n = n; pp.K = Kdim; pp.permute = 0; pp.act_blocks = n;
+    pp.n = n; pp.K = Kdim; pp.act_blocks = n;
     pp.ld_in = (long long)ldact; pp.ld_out = pl.ld_act;
     pp.in = reinterpret_cast<const __nv_bfloat16*>(act); pp.out = act16; pp.tok_inv_scale = tok;
     pp.alpha = alpha; pp.alpha_count = (long long)bcq_alpha_count(d_out, d_in, q, g); pp.hdr = hdr;
