@@ -270,8 +270,10 @@ DalphaPlan plan_dalpha(int d_out, int d_in, int g, int n) {
     const int sms = sm_count();
     pl.m_tiles = ceil_div(d_out, kBlockM);
     pl.num_kb = ceil_div(n, kBlockK);
-    pl.TN = 256;
-    if (d_in <= 128 || pl.m_tiles * ceil_div(d_in, 256) < sms) pl.TN = 128;
+    // The UMMA-issuing thread needs about 0.3 us per 64-token stage whatever the tile width, more
+    // than a 128 x 128 x 64 UMMA group takes to execute, so wide tiles (and a token split when
+    // they do not fill the SMs) beat twice as many narrow ones.
+    pl.TN = (d_in <= 128) ? 128 : 256;
     pl.HN = pl.TN / 2;
     pl.n_tiles = ceil_div(d_in, pl.TN);
     pl.n_subtiles = pl.n_tiles * 2;
