@@ -1405,14 +1405,13 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     if (n <= 32) tn = 32;
     else if (n <= 64) tn = 64;
     else if (n <= 128) tn = 128;
-    else {
-        tn = 256;
-        if (pl.m_tiles * ceil_div(n, 256) < sms) tn = 128;
-    }
+    else tn = 256;  // the expansion and the UMMA issue cost the same per stage whatever the width
     pl.TN = tn;
     pl.n_tiles = ceil_div(n, tn);
     const int tiles = pl.m_tiles * pl.n_tiles;
-    int splits = sms / tiles;
+    // The K split goes through fp32 partials, a slower epilogue and a second kernel: only for
+    // problems that would otherwise leave most of the SMs idle.
+    int splits = (4 * tiles <= sms) ? sms / tiles : 1;
     if (splits < 1) splits = 1;
     const int max_splits = (pl.num_kb + 3) / 4;  // at least 4 K blocks per CTA
     if (splits > max_splits) splits = max_splits;
