@@ -366,11 +366,15 @@ template <int VPL>
 __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
     __shared__ uint32_t red[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if ((int)blockIdx.x >= p.act_blocks + p.amax_blocks) {
+    // roles by block id: tokens, then max|alpha|, then the regrouping blocks.  The hardware starts
+    // blocks in index order, and the short, latency-bound regrouping blocks should not queue
+    // behind the register-heavy token blocks, so the ids run backwards.
+    const int bid = (int)gridDim.x - 1 - (int)blockIdx.x;
+    if (bid >= p.act_blocks + p.amax_blocks) {
         // ---- regroup a block of 128 rows x 32 columns (plane words or scales) of one plane:
         // coalesced reads into shared memory, then coalesced writes of the stage chunks
         __shared__ uint32_t tile[128][33];
-        int b = (int)blockIdx.x - p.act_blocks - p.amax_blocks;
+        int b = bid - p.act_blocks - p.amax_blocks;
         const bool is_alpha = b >= p.bits_blocks;
         if (is_alpha) b -= p.bits_blocks;
         const int cblks = is_alpha ? p.alpha_cblk : p.bits_cblk;
@@ -432,11 +436,11 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         }
         return;
     }
-    if ((int)blockIdx.x >= p.act_blocks) {
+    if (bid >= p.act_blocks) {
         // ---- max |alpha| of this block's share of the scales
         const long long nb = p.amax_blocks;
         uint32_t m = 0u;
-        for (long long o = ((long long)blockIdx.x - p.act_blocks) * 256 + threadIdx.x; o < p.alpha_count;
+        for (long long o = ((long long)bid - p.act_blocks) * 256 + threadIdx.x; o < p.alpha_count;
              o += nb * 256)
             m = max(m, __float_as_uint(__ldg(p.alpha + o)) & 0x7FFFFFFFu);
 #pragma unroll
@@ -446,12 +450,12 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         if (threadIdx.x == 0) {
 #pragma unroll
             for (int w = 0; w < 8; ++w) m = max(m, red[w]);
-            p.hdr->block_max[blockIdx.x - p.act_blocks] = m;
-            if ((int)blockIdx.x == p.act_blocks) p.hdr->nblocks = (uint32_t)nb;
+            p.hdr->block_max[bid - p.act_blocks] = m;
+            if (bid == p.act_blocks) p.hdr->nblocks = (uint32_t)nb;
         }
         return;
     }
-    const int t = blockIdx.x * kPrepTokensPerBlock + warp;
+    const int t = bid * kPrepTokensPerBlock + warp;
     if (t >= p.n) return;
     const uint4* src = reinterpret_cast<const uint4*>(p.in + (long long)t * p.ld_in);
     uint4* dst = reinterpret_cast<uint4*>(p.out + (long long)t * p.ld_out);
