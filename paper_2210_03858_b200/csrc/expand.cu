@@ -608,24 +608,26 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(ctl.aready + 8 * s, kPfGroupWarps + 1);  // both operands: the worker warps and the activation tile
-            ptx::mbar_init(ctl.empty + 8 * s, 1);
+    if (warp == 0) {
+        // the barriers are initialised by the lanes of one warp side by side (one after the other
+        // they cost a few tenths of a microsecond before any copy can start)
+        if (lane < STAGES) {
+            ptx::mbar_init(ctl.aready + 8 * lane, kPfGroupWarps + 1);  // both operands: the worker warps and the activation tile
+            ptx::mbar_init(ctl.empty + 8 * lane, 1);
+        } else if (lane >= 8 && lane < 8 + AUXS) {
+            ptx::mbar_init(wfull + 8 * (lane - 8), 1 + p.alpha_parts);  // plane words; each part of the scales
+            ptx::mbar_init(wempty + 8 * (lane - 8), kPfGroupWarps);
+        } else if (lane >= 16 && lane < 18) {
+            ptx::mbar_init(ctl.accum + 8 * (lane - 16), 1);
+            ptx::mbar_init(acc_empty + 8 * (lane - 16), kPfEpiWarps);
+        } else if (lane == 18) {
+            ptx::mbar_init(ctl.spare, 1);
+            *ctl.abort_flag = 0;
+        } else if (lane == 19) {
+            ptx::prefetch_tmap(&tmap_b);
+            if (p.fast_epi) ptx::prefetch_tmap(&tmap_out);
         }
-        for (int a = 0; a < AUXS; ++a) {
-            ptx::mbar_init(wfull + 8 * a, 1 + p.alpha_parts);  // plane words; each part of the scales
-            ptx::mbar_init(wempty + 8 * a, kPfGroupWarps);
-        }
-        for (int a = 0; a < 2; ++a) {
-            ptx::mbar_init(ctl.accum + 8 * a, 1);
-            ptx::mbar_init(acc_empty + 8 * a, kPfEpiWarps);
-        }
-        ptx::mbar_init(ctl.spare, 1);
-        *ctl.abort_flag = 0;
         ptx::fence_mbar_init();
-        ptx::prefetch_tmap(&tmap_b);
-        if (p.fast_epi) ptx::prefetch_tmap(&tmap_out);
     }
     if (warp == kPfMmaWarp) {
         ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);

@@ -37,9 +37,6 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ct
     uint32_t spins = 0;
     while (true) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-#ifdef BCQ_WAIT_SLEEP_NS
-        __nanosleep(BCQ_WAIT_SLEEP_NS);
-#endif
         if ((++spins & 7u) == 0u) {
             if (*ctl.abort_flag) return false;
             if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
