@@ -1557,9 +1557,10 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     pp.act_blocks = tok_blocks;
     const unsigned pgrid = (unsigned)(tok_blocks + ablocks + pp.bits_blocks + alpha_tr_blocks);
     const int nvec = (Kdim + 7) / 8;
+    // Rows of up to 1024 elements stay in registers between the two passes over them.  Longer
+    // rows are read twice instead (the second time from L2): holding them would cost so many
+    // registers that the grid no longer fits on the SMs in one wave.
     if (nvec <= 32 * 4) prepare_kernel<4><<<pgrid, 256, 0, s>>>(pp);
-    else if (nvec <= 32 * 8) prepare_kernel<8><<<pgrid, 256, 0, s>>>(pp);
-    else if (nvec <= 32 * 16) prepare_kernel<16><<<pgrid, 256, 0, s>>>(pp);
     else prepare_kernel<0><<<pgrid, 256, 0, s>>>(pp);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
