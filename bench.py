@@ -169,28 +169,32 @@ def run_gpu(args):
             dY = torch.randn((TOKENS, d_out), generator=gen, device=dev, dtype=torch.float32).bfloat16()
             layers.append(dict(d_in=d_in, d_out=d_out, bits=bits, alpha=alpha, X=X, dY=dY,
                                dalpha=torch.zeros_like(alpha)))
-    # outputs and workspaces: one set per shape and per operation, so that the three operations of
-    # a step can run on three streams at once
+    # outputs and workspaces: one set per shape, per operation and per chain, so that the operations
+    # of a step can run on several streams at once
+    chains = max(1, args.chains)
+    for i, l in enumerate(layers):
+        l["chain"] = i % chains
     bufs = {}
     out_dtype = torch.bfloat16 if args.out_bf16 else torch.float32
     for _, d_in, d_out in LINEARS:
         def ws(op):
             return torch.empty(max(16, bcq.workspace_bytes(op, d_out, d_in, Q, d_in, TOKENS)), dtype=torch.uint8, device=dev)
-        bufs[(d_in, d_out)] = dict(Y=torch.empty((TOKENS, d_out), device=dev, dtype=out_dtype),
-                                   dX=torch.empty((TOKENS, d_in), device=dev, dtype=out_dtype),
-                                   ws_fwd=ws(bcq.OP_FWD), ws_dx=ws(bcq.OP_BWD_X), ws_da=ws(bcq.OP_BWD_ALPHA))
+        for c in range(chains):
+            bufs[(d_in, d_out, c)] = dict(Y=torch.empty((TOKENS, d_out), device=dev, dtype=out_dtype),
+                                          dX=torch.empty((TOKENS, d_in), device=dev, dtype=out_dtype),
+                                          ws_fwd=ws(bcq.OP_FWD), ws_dx=ws(bcq.OP_BWD_X), ws_da=ws(bcq.OP_BWD_ALPHA))
     flat_dalpha = torch.zeros(sum(l["dalpha"].numel() for l in layers), device=dev) if world > 1 else None
 
     def op_fwd(l):
-        b = bufs[(l["d_in"], l["d_out"])]
+        b = bufs[(l["d_in"], l["d_out"], l["chain"])]
         bcq.linear_fwd(l["X"], l["bits"], l["alpha"], l["d_in"], l["d_in"], out=b["Y"], ws=b["ws_fwd"])
 
     def op_da(l):
-        b = bufs[(l["d_in"], l["d_out"])]
+        b = bufs[(l["d_in"], l["d_out"], l["chain"])]
         bcq.linear_bwd_alpha(l["dY"], l["X"], l["bits"], l["d_in"], l["d_in"], out=l["dalpha"], ws=b["ws_da"])
 
     def op_dx(l):
-        b = bufs[(l["d_in"], l["d_out"])]
+        b = bufs[(l["d_in"], l["d_out"], l["chain"])]
         bcq.linear_bwd_x(l["dY"], l["bits"], l["alpha"], l["d_in"], l["d_in"], out=b["dX"], ws=b["ws_dx"])
 
     OPS = (("fwd", op_fwd), ("bwd_alpha", op_da), ("bwd_x", op_dx))
@@ -199,24 +203,25 @@ def run_gpu(args):
         for _, fn in OPS:
             fn(l)
 
-    # the dX chain is the longest of the three, so its stream gets the higher priority
-    side = [torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev, priority=-1)]
+    # one stream per (operation, chain); the dX chains are the longest, so theirs get the higher priority
+    streams = {}
+    for name, _ in OPS:
+        for c in range(chains):
+            streams[(name, c)] = torch.cuda.Stream(device=dev, priority=-1 if name == "bwd_x" else 0)
 
     def enqueue_step():
         # the linears are independent problems, and within one linear dalpha and dX only share their
-        # inputs: forward, dalpha and dX are enqueued as three chains on three streams
+        # inputs: forward, dalpha and dX of the linears of a chain are three queues on three streams
         cur = torch.cuda.current_stream()
-        for s_ in side:
+        for s_ in streams.values():
             s_.wait_stream(cur)
-        for l in layers:
-            op_fwd(l)
-        with torch.cuda.stream(side[0]):
-            for l in layers:
-                op_da(l)
-        with torch.cuda.stream(side[1]):
-            for l in layers:
-                op_dx(l)
-        for s_ in side:
+        for name, fn in OPS:
+            for c in range(chains):
+                with torch.cuda.stream(streams[(name, c)]):
+                    for l in layers:
+                        if l["chain"] == c:
+                            fn(l)
+        for s_ in streams.values():
             cur.wait_stream(s_)
 
     # warm up outside capture (also resolves lazy CUDA state), then capture one step as a CUDA graph
@@ -362,7 +367,7 @@ def run_gpu(args):
             "config": {"workload": WORKLOAD, "layers": LAYERS, "tokens_per_gpu": TOKENS, "q": Q, "g": "d_in",
                        "l2": "a step touches ~1.5 GB of distinct inputs, far more than the 126 MB L2",
                        "outputs": "bf16" if args.out_bf16 else "fp32",
-                       "launch": ("one CUDA graph per step, " if args.graph else "") + "forward / dalpha / dX on three streams (dX at high priority)",
+                       "launch": ("one CUDA graph per step, " if args.graph else "") + "forward / dalpha / dX on %d streams (dX at high priority)" % (3 * chains),
                        "parallelism": "dp%d" % world, "quantize_ms_once": quant_ms},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
             "cpu_baseline": cpu_baseline}
@@ -416,6 +421,9 @@ def main():
     ap.add_argument("--no-decode", dest="decode", action="store_false")
     ap.add_argument("--no-graph", dest="graph", action="store_false", help="launch every kernel from the host each step")
     ap.add_argument("--out-fp32", dest="out_bf16", action="store_false", help="fp32 Y and dX instead of bf16")
+    ap.add_argument("--chains", type=int, default=3,
+                    help="independent chains per operation: the linears of a step are dealt round-robin to this many "
+                         "streams (each with its own outputs and workspaces) for each of forward, dalpha and dX")
     ap.add_argument("--timed-only", action="store_true",
                     help="warm-up and timed steps only (no per-operation, end-to-end, CPU or decode legs): the command to profile")
     args = ap.parse_args()
