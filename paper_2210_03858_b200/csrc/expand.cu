@@ -1497,7 +1497,11 @@ bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const Ex
     auto kern = expand_gemm_kernel<MODE, TN, QM>;
     BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
-    const int grid = tiles < sm_count() ? tiles : sm_count();  // persistent: one CTA per SM
+    // persistent, at most one CTA per SM; with more tiles than SMs every CTA gets the same number of
+    // tiles (as many as the busiest would get anyway): fewer CTAs pay the prologue, more epilogues
+    // overlap the next tile's main loop, and the SMs left over can run other kernels
+    const int per_cta = ceil_div(tiles, sm_count());
+    const int grid = ceil_div(tiles, per_cta);
     kern<<<grid, kPfThreads, pl.smem, stream>>>(tm, tmo, p);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
