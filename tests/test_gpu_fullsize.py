@@ -72,8 +72,16 @@ def test_prefill_layer_sampled(workload, n, d_in, d_out, q, g):
     # which max over the samples is a (smaller, hence stricter) stand-in
     ref = oracle.fwd_at(X, hb, ha, d_in, g, t, j)
     _check_sampled(Y, ref, (t, j), np.abs(ref).max())
-    ref = oracle.bwd_x_at(dY, hb, ha, d_in, g, t, k)
-    _check_sampled(dX, ref, (t, k), np.abs(ref).max())
+    ref_dx = oracle.bwd_x_at(dY, hb, ha, d_in, g, t, k)
+    _check_sampled(dX, ref_dx, (t, k), np.abs(ref_dx).max())
+    # bf16 outputs, as bench.py launches the layer (another epilogue: one more rounding, 2^-8)
+    Yb = bcq.linear_fwd(Xd, bits, alpha, d_in, g, out_dtype=torch.bfloat16).float().cpu().numpy()
+    dXb = bcq.linear_bwd_x(dYd, bits, alpha, d_in, g, out_dtype=torch.bfloat16).float().cpu().numpy()
+    assert np.abs(Yb[(t, j)] - ref).max() <= (TOL + 2.0 ** -8) * np.abs(ref).max()
+    assert np.abs(dXb[(t, k)] - ref_dx).max() <= (TOL + 2.0 ** -8) * np.abs(ref_dx).max()
+    # and the whole bf16 output against the fp32 one: a misplaced tile would show here
+    assert np.abs(Yb - Y).max() <= 2.0 ** -7 * np.abs(Y).max()
+    assert np.abs(dXb - dX).max() <= 2.0 ** -7 * np.abs(dX).max()
     jj = j[: NS // 8]
     ref = oracle.bwd_alpha_at(dY, X, hb, d_in, g, i, jj, c)
     _check_sampled(dA, ref, (i, jj, c), np.abs(ref).max())
