@@ -58,7 +58,8 @@ typedef enum {
     BCQ_OP_FWD = 1,
     BCQ_OP_DECODE = 2,
     BCQ_OP_BWD_X = 3,
-    BCQ_OP_BWD_ALPHA = 4
+    BCQ_OP_BWD_ALPHA = 4,
+    BCQ_OP_DECODE_PACKED = 5
 } bcq_op;
 
 /* ------------------------------------------------------------------ sizes (host only) */
@@ -162,6 +163,38 @@ bcq_status bcq_linear_decode_noalloc(int d_out, int d_in, int q, int g, int n, c
                                      size_t ldx, const uint32_t* bits, const float* alpha,
                                      const float* bias, void* Y, size_t ldy, int y_dtype,
                                      void* stream);
+
+/* Decode from a packed copy of the frozen weights.
+ *
+ * At inference both B and alpha are fixed (Section "Inference Speed": a small-batch layer costs
+ * what moving its weights costs), so whatever does not depend on the activations can be done
+ * once.  bcq_decode_pack rewrites a quantized matrix (q <= 4) into the order and encoding the
+ * decode kernel consumes:
+ *   - per weight the index of its level among the 2^q sums +-alpha_1 .. +-alpha_q of its
+ *     (row, group), q bits per weight as in `bits`;
+ *   - per (row, group) the eight fp16 levels sum_i +-alpha_i (for q = 4 those with b_4 = +1; the
+ *     others are their negatives), 16 bytes, multiplied by a power of two per row that brings
+ *     q * max|alpha| of the row to [2^13, 2^14) -- the values bcq_linear_decode forms on the fly;
+ *   - per row that power of two, and one arrival counter per tile of 128 rows.
+ * The pack is bcq_decode_pack_bytes() bytes (0 for an unsupported shape; about the size of bits
+ * plus alpha), 128-byte aligned, caller-owned.  q > 4 gives BCQ_ERR_UNSUPPORTED: use
+ * bcq_linear_decode.  If alpha changes, pack again. */
+size_t bcq_decode_pack_bytes(int d_out, int d_in, int q, int g);
+bcq_status bcq_decode_pack(int d_out, int d_in, int q, int g, const uint32_t* bits, const float* alpha,
+                           void* pack, size_t pack_bytes, void* stream);
+
+/* Y = X W_hat^T (+ bias) for 1 <= n <= 16 tokens from a pack (Eq. 2; same arithmetic as
+ * bcq_linear_decode: fp16 levels, bf16 activations scaled per token by a power of two, fp32
+ * accumulation).  One kernel: the 128-row x 128-column pieces of the matrix are dealt evenly to
+ * one CTA per SM; where two CTAs share a row tile the partial sums go through `ws`
+ * (bcq_workspace_bytes(BCQ_OP_DECODE_PACKED, ...) bytes, may be 0) and are added in a fixed order,
+ * so the result is the same in every run.
+ * The pack is not const: the call uses its arrival counters and leaves them zero again.  Calls
+ * that use the same pack must not overlap on the GPU.  After BCQ_ERR_DEVICE_TIMEOUT (see
+ * bcq_device_timeout_flag) write the pack again. */
+bcq_status bcq_linear_decode_packed(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                                    void* pack, const float* bias, void* Y, size_t ldy, int y_dtype,
+                                    void* ws, size_t ws_bytes, void* stream);
 
 /* Input gradient (Eq. 3):  dX[t][k] = sum_j dY[t][j] * W_hat[j][k],  W_hat as in Eq. 1.
  *   dY in : bf16 [n][lddy];   dX out: dx_dtype [n][lddx], lddx >= d_in. */

@@ -17,14 +17,15 @@ LIB_PATH = os.path.join(_HERE, "libbcq_b200.so")
 
 OK = 0
 F32, BF16 = 0, 1
-OP_QUANTIZE, OP_FWD, OP_DECODE, OP_BWD_X, OP_BWD_ALPHA = 0, 1, 2, 3, 4
+OP_QUANTIZE, OP_FWD, OP_DECODE, OP_BWD_X, OP_BWD_ALPHA, OP_DECODE_PACKED = 0, 1, 2, 3, 4, 5
 
 # every symbol include/bcq.h declares
 SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_count",
            "bcq_payload_bits", "bcq_workspace_bytes", "bcq_quantize", "bcq_dequantize",
            "bcq_linear_fwd", "bcq_linear_decode", "bcq_linear_bwd_x", "bcq_linear_bwd_alpha",
            "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag",
-           "bcq_kernel_launches", "bcq_linear_decode_noalloc")
+           "bcq_kernel_launches", "bcq_linear_decode_noalloc", "bcq_decode_pack_bytes",
+           "bcq_decode_pack", "bcq_linear_decode_packed")
 
 
 class BcqError(RuntimeError):
@@ -68,6 +69,12 @@ def lib() -> C.CDLL:
         l.bcq_linear_decode.argtypes = l.bcq_linear_fwd.argtypes
         l.bcq_linear_decode_noalloc.restype = i
         l.bcq_linear_decode_noalloc.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, vp, sz, i, vp]
+        l.bcq_decode_pack_bytes.restype = sz
+        l.bcq_decode_pack_bytes.argtypes = [i, i, i, i]
+        l.bcq_decode_pack.restype = i
+        l.bcq_decode_pack.argtypes = [i, i, i, i, vp, vp, vp, sz, vp]
+        l.bcq_linear_decode_packed.restype = i
+        l.bcq_linear_decode_packed.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_bwd_x.restype = i
         l.bcq_linear_bwd_x.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_bwd_alpha.restype = i
@@ -199,6 +206,35 @@ def linear_decode(X, bits, alpha, d_in: int, g: int, bias=None, out=None, out_dt
     """bcq_linear_decode: same as linear_fwd for 1..16 tokens."""
     return _fwd(lib().bcq_linear_decode, OP_DECODE, "bcq_linear_decode", X, bits, alpha, d_in, g,
                 bias, out, out_dtype, ws)
+
+
+def decode_pack(bits, alpha, d_in: int, g: int):
+    """bcq_decode_pack: the frozen (bits, alpha) of a layer rewritten for bcq_linear_decode_packed
+    (q <= 4).  Returns the pack as a uint8 tensor."""
+    torch = _torch()
+    q, d_out, _ = bits.shape
+    nbytes = lib().bcq_decode_pack_bytes(d_out, d_in, q, g)
+    if nbytes == 0:
+        raise BcqError(-4, "bcq_decode_pack_bytes")
+    pack = torch.empty(nbytes, dtype=torch.uint8, device=bits.device)
+    _check(lib().bcq_decode_pack(d_out, d_in, q, g, _ptr(bits), _ptr(alpha), _ptr(pack), nbytes,
+                                 _stream()), "bcq_decode_pack")
+    return pack
+
+
+def linear_decode_packed(X, pack, d_out: int, d_in: int, q: int, g: int, bias=None, out=None,
+                         out_dtype=None, ws=None):
+    """bcq_linear_decode_packed: X bf16 [n][d_in], n <= 16 -> Y [n][d_out] from a pack."""
+    torch = _torch()
+    assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    n = X.shape[0]
+    if out is None:
+        out = torch.empty((n, d_out), dtype=out_dtype or torch.float32, device=X.device)
+    ws, ws_bytes = _ws(OP_DECODE_PACKED, d_out, d_in, q, g, n, ws, X.device)
+    _check(lib().bcq_linear_decode_packed(d_out, d_in, q, g, n, _ptr(X), X.stride(0), _ptr(pack),
+                                          _ptr(bias), _ptr(out), out.stride(0), _dtype_code(out),
+                                          _ptr(ws), ws_bytes, _stream()), "bcq_linear_decode_packed")
+    return out
 
 
 NOALLOC_SCRATCH_BYTES = 2 << 20

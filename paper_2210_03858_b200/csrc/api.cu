@@ -52,12 +52,14 @@ extern "C" int bcq_last_cuda_error(void) { return bcq::t_last_cuda_error; }
 extern "C" bcq_status bcq_device_timeout_flag(int* flag_out, int reset) {
     if (flag_out == nullptr) return BCQ_ERR_NULL;
     BCQ_CUDA_TRY(cudaDeviceSynchronize());
-    int a = 0, b = 0;
+    int a = 0, b = 0, c = 0;
     bcq_status st = bcq::expand_timeout_flag(&a, reset);
     if (st != BCQ_OK) return st;
     st = bcq::dalpha_timeout_flag(&b, reset);
     if (st != BCQ_OK) return st;
-    *flag_out = a != 0 ? a : b;
+    st = bcq::decode_timeout_flag(&c, reset);
+    if (st != BCQ_OK) return st;
+    *flag_out = a != 0 ? a : (b != 0 ? b : c);
     return BCQ_OK;
 }
 
@@ -69,6 +71,7 @@ extern "C" size_t bcq_workspace_bytes(int op, int d_out, int d_in, int q, int g,
         case BCQ_OP_DECODE: return n > 16 ? 0 : bcq::decode_workspace_bytes(d_out, d_in, q, g, n);
         case BCQ_OP_BWD_X: return bcq::bwd_x_workspace_bytes(d_out, d_in, q, g, n);
         case BCQ_OP_BWD_ALPHA: return bcq::bwd_alpha_workspace_bytes(d_out, d_in, q, g, n);
+        case BCQ_OP_DECODE_PACKED: return n > 16 ? 0 : bcq::decode_packed_workspace_bytes(d_out, d_in, q, g, n);
         default: return 0;
     }
 }

@@ -30,6 +30,7 @@
 #include <mutex>
 
 #include "gemm_common.cuh"
+#include "lut.cuh"
 
 namespace {
 
@@ -40,60 +41,6 @@ __device__ int g_timeout_flag = 0;
 enum { MODE_FWD = 0, MODE_BWDX = 1 };
 enum { QM_LUT3 = 0, QM_LUT4 = 1, QM_GENERIC = 2 };
 constexpr int kPrefetch = 3;  // stages between the global loads of a task and its use
-
-// ------------------------------------------------------------------------------------------
-// small device helpers
-// ------------------------------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t c) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
-__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
-    __half2 h = __floats2half2_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-
-// 2^e as a float, e clamped to the normal range.
-__device__ __forceinline__ float pow2f(int e) {
-    e = max(-126, min(127, e));
-    return __uint_as_float((uint32_t)(e + 127) << 23);
-}
-
-// Exponent of a positive finite float given by its bits (0 for zero / subnormal input).
-__device__ __forceinline__ int exponent_of_bits(uint32_t fbits) {
-    const int be = (int)((fbits >> 23) & 0xFFu);
-    return be == 0 ? -127 : be - 127;
-}
-
-// Power of two that brings a magnitude with exponent `e` to [2^target, 2^(target+1)).
-__device__ __forceinline__ int shift_for(int e, int target) {
-    if (e <= -127 || e >= 128) return 0;  // zero, subnormal, inf or nan: leave alone
-    return max(-100, min(100, target - e));
-}
-
-// Byte-wise lookup table of eight fp16 levels: tl* low bytes, th* high bytes; *0 = levels 0..3.
-struct Lut {
-    uint32_t tl0, tl1, th0, th1;
-};
-
-// Level s (bit i of s set <=> plane i is +1) = base + sum_{i<3} (+-a_i).
-__device__ __forceinline__ Lut build_lut(float a0, float a1, float a2, float base) {
-    const float t0 = base - a0, t1 = base + a0;
-    const float u0 = t0 - a1, u1 = t1 - a1, u2 = t0 + a1, u3 = t1 + a1;
-    const uint32_t p0 = pack_half2(u0 - a2, u1 - a2);
-    const uint32_t p1 = pack_half2(u2 - a2, u3 - a2);
-    const uint32_t p2 = pack_half2(u0 + a2, u1 + a2);
-    const uint32_t p3 = pack_half2(u2 + a2, u3 + a2);
-    Lut t;
-    t.tl0 = prmt(p0, p1, 0x6420u);
-    t.th0 = prmt(p0, p1, 0x7531u);
-    t.tl1 = prmt(p2, p3, 0x6420u);
-    t.th1 = prmt(p2, p3, 0x7531u);
-    return t;
-}
 
 // 16 weights of one row (bits 0..15 of the plane words w0..w3) through the lookup table, stored
 // as two 16-byte chunks (slots chunk0, chunk0 + 1) of the 128-byte line at `line` (swizzle key
@@ -516,6 +463,7 @@ struct ExpandParams {
     long long ldo;
     int out_bf16;
     int fast_epi;                // bf16 output written by TMA stores (aligned base and pitch, no K split)
+    int helpers;                 // the worker warps share the epilogue of a CTA's last tile (see run_expand)
     float* partial;              // [splits][n][Mdim] when splits > 1
 };
 
@@ -917,7 +865,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             }
             gi = (gi + iters) % kPfGroups;
         }
-        if (p.fast_epi && ok && (int)blockIdx.x < num_tiles) {
+        if (p.helpers && ok && (int)blockIdx.x < num_tiles) {
             // share the epilogue of this CTA's last tile.  Its operand slots are free once the
             // accumulator is complete, so each warp stages its boxes in 1 KiB of the first slots.
             const int lt = (num_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x;
@@ -995,7 +943,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
                     b4[i] = (MODE == MODE_FWD && p.bias != nullptr && m0w + g + 8 * i < p.Mdim) ? __ldg(p.bias + m0w + g + 8 * i) : 0.0f;
-                const int cstep = is_last_tile(tile) ? 16 * kPfHelpers : 16;  // the workers take the other boxes
+                const int cstep = (p.helpers && is_last_tile(tile)) ? 16 * kPfHelpers : 16;  // the workers take the other boxes
 #pragma unroll 1
                 for (int col = 0; col < TN; col += cstep) {
                     if (t0 + col >= p.n || m0w >= p.Mdim) break;  // uniform in the warp
@@ -1126,16 +1074,16 @@ struct DecodeParams {
 constexpr int kDecTN = 16;
 constexpr int kDecStages = 4;
 
-// Scale of one weight row in decode: the scales of the row's first groups inside the CTA's K slice
-// (at most four) are sampled; their maximum times q is brought to 2^9, which leaves a factor of
-// 64 of headroom for larger scales further along the row before fp16 would overflow.
+// Scale of one weight row in decode: the largest |alpha| of the row over every plane and every
+// group inside the CTA's K slice, times q (a bound on any level sum_i +-alpha_i), is brought to
+// [2^13, 2^14), so no level of the slice can leave the fp16 range.
 __device__ __forceinline__ int decode_row_shift(const float* __restrict__ alpha, long long plane_alpha, int G,
                                                 int q, int j, int c_lo, int c_hi) {
     uint32_t am = 0u;
     for (int i = 0; i < q; ++i)
-        for (int c = c_lo; c <= min(c_hi, c_lo + 3); ++c)
+        for (int c = c_lo; c <= c_hi; ++c)
             am = max(am, __float_as_uint(__ldg(alpha + i * plane_alpha + (long long)j * G + c)) & 0x7FFFFFFFu);
-    return shift_for(exponent_of_bits(__float_as_uint(__uint_as_float(am) * (float)q)), 9);
+    return shift_for(exponent_of_bits(__float_as_uint(__uint_as_float(am) * (float)q)), 13);
 }
 
 template <int QM>
@@ -1587,6 +1535,11 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
         st = make_tmap_out_bf16(&tmo, out, Mdim, n, ldo);
         if (st != BCQ_OK) return st;
     }
+    // The workers find the last tile's accumulator by barrier parity alone.  They run at most
+    // `stages` pipeline stages ahead of the tensor core, so the parity is unambiguous only if
+    // two tiles are longer than that: then the accumulator's previous use (two tiles back) is
+    // certain to be complete when a worker has finished the last tile's stages.
+    p.helpers = (p.fast_epi && 2 * pl.num_kb >= pl.stages + 2) ? 1 : 0;
     switch (pl.TN) {
         case 32: st = launch_expand_q<MODE, 32>(tm, tmo, p, pl, s); break;
         case 64: st = launch_expand_q<MODE, 64>(tm, tmo, p, pl, s); break;

@@ -31,12 +31,22 @@ struct Ctl {
 
 // Waits for the phase with the given parity.  Gives up after kWaitLimitNs (or as soon as another
 // thread of the CTA gave up), records `code` in the device flag and returns false.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl& ctl, int code) {
+// Between polls the warp sleeps for `nap_ns`: a warp that spins on try_wait keeps winning issue
+// slots from the warps that do the work (measured: about half of all instructions a kernel issued
+// were polls), while a sleeping warp costs nothing; the price is up to nap_ns of extra latency
+// when the phase completes, so waits on the critical path take a short nap and long, off-path
+// waits (an epilogue waiting for a whole tile) a longer one.
+#ifndef BCQ_NAP_NS
+#define BCQ_NAP_NS 128u
+#endif
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, const Ctl& ctl, int code,
+                                         uint32_t nap_ns = BCQ_NAP_NS) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = ptx::globaltimer_ns();
     uint32_t spins = 0;
     while (true) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
+        __nanosleep(nap_ns);
         if ((++spins & 7u) == 0u) {
             if (*ctl.abort_flag) return false;
             if (ptx::globaltimer_ns() - t0 > kWaitLimitNs) {
@@ -179,11 +189,13 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // per-TU device timeout flags
 bcq_status expand_timeout_flag(int* flag_out, int reset);
 bcq_status dalpha_timeout_flag(int* flag_out, int reset);
+bcq_status decode_timeout_flag(int* flag_out, int reset);
 
 // workspace sizes (defined next to the kernels that use them)
 size_t fwd_workspace_bytes(int d_out, int d_in, int q, int g, int n);
 size_t decode_workspace_bytes(int d_out, int d_in, int q, int g, int n);
 size_t bwd_x_workspace_bytes(int d_out, int d_in, int q, int g, int n);
 size_t bwd_alpha_workspace_bytes(int d_out, int d_in, int q, int g, int n);
+size_t decode_packed_workspace_bytes(int d_out, int d_in, int q, int g, int n);
 
 }  // namespace bcq

@@ -69,6 +69,30 @@ def sample_indices(count: int, bounds, key) -> list:
     return [rng.integers(0, b, size=count, dtype=np.int64) for b in bounds]
 
 
+def stratified_indices(rows: int, cols: int, tile_rows: int, tile_cols: int, per_tile: int, key) -> list:
+    """``per_tile`` (row, column) positions drawn uniformly inside every tile_rows x tile_cols tile
+    of a rows x cols matrix (edge tiles are clipped), so that no tile of an output is left
+    without a sampled value.  Returns [row indices, column indices]."""
+    rng = rng_for(*key, ROLE_IDX)
+    rr, cc = [], []
+    for r0 in range(0, rows, tile_rows):
+        rh = min(tile_rows, rows - r0)
+        for c0 in range(0, cols, tile_cols):
+            cw = min(tile_cols, cols - c0)
+            rr.append(r0 + rng.integers(0, rh, size=per_tile, dtype=np.int64))
+            cc.append(c0 + rng.integers(0, cw, size=per_tile, dtype=np.int64))
+    return [np.concatenate(rr), np.concatenate(cc)]
+
+
+def line_indices(rows: int, cols: int, row_lines, col_lines) -> list:
+    """Every position of the given whole rows and whole columns of a rows x cols matrix."""
+    rr = [np.repeat(np.asarray(row_lines, dtype=np.int64), cols)]
+    cc = [np.tile(np.arange(cols, dtype=np.int64), len(row_lines))]
+    rr.append(np.tile(np.arange(rows, dtype=np.int64), len(col_lines)))
+    cc.append(np.repeat(np.asarray(col_lines, dtype=np.int64), rows))
+    return [np.concatenate(rr), np.concatenate(cc)]
+
+
 # ----------------------------------------------------------------------------------------
 # Workloads: (name, d_in, d_out) of the quantized linears of one Transformer block.
 # ----------------------------------------------------------------------------------------

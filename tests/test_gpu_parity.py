@@ -216,6 +216,148 @@ def test_decode_matches_oracle(n, d_in, d_out, q, g):
     assert rel_err(Y.cpu().numpy(), ref) <= TOL
 
 
+# --------------------------------------------------------------------------- tile-schedule corners
+
+@pytest.mark.parametrize("n", [1, 17, 31, 32])
+def test_fwd_and_bwd_x_with_few_tokens(n):
+    # the prefill entry points accept any n >= 1; n <= 32 takes the narrowest token tile
+    d_in, d_out, q, g = 640, 384, 3, 128
+    _, X, dY, bits, alpha, _, _ = make_case(700 + n, n, d_in, d_out, q, g)
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref_y = oracle.fwd(X, bits, alpha, d_in, g)
+    ref_dx = oracle.bwd_x(dY, bits, alpha, d_in, g)
+    for dt, tol in ((torch.float32, TOL), (torch.bfloat16, TOL + 2.0 ** -8)):
+        assert rel_err(bcq.linear_fwd(Xd, bd, ad, d_in, g, out_dtype=dt).float().cpu().numpy(), ref_y) <= tol
+        assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=dt).float().cpu().numpy(), ref_dx) <= tol
+
+
+@pytest.mark.parametrize("d_in", [64, 128, 192])
+def test_many_tiles_per_cta_with_short_k(d_in):
+    # 320 output tiles of 128 x 256 on 148 SMs: every persistent CTA walks three tiles, so both
+    # accumulators are reused (second phase of their barriers) and, with K this short, the worker
+    # warps are far ahead of the tensor core when they reach the last tile's epilogue
+    n, d_out, q, g = 4096, 2560, 3, 64
+    _, X, dY, bits, alpha, _, _ = make_case(800 + d_in, n, d_in, d_out, q, g)
+    Xd, _, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    Yb = bcq.linear_fwd(Xd, bd, ad, d_in, g, out_dtype=torch.bfloat16)
+    Yb2 = bcq.linear_fwd(Xd, bd, ad, d_in, g, out_dtype=torch.bfloat16)
+    assert torch.equal(Yb, Yb2)
+    assert rel_err(Yb.float().cpu().numpy(), ref) <= TOL + 2.0 ** -8
+    assert rel_err(bcq.linear_fwd(Xd, bd, ad, d_in, g).cpu().numpy(), ref) <= TOL
+
+
+def test_bwd_x_many_tiles_per_cta_with_short_k():
+    n, d_in, d_out, q, g = 4096, 2560, 64, 4, 128
+    _, X, dY, bits, alpha, _, _ = make_case(811, n, d_in, d_out, q, g)
+    _, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.bwd_x(dY, bits, alpha, d_in, g)
+    assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=torch.bfloat16).float().cpu().numpy(),
+                   ref) <= TOL + 2.0 ** -8
+    assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g).cpu().numpy(), ref) <= TOL
+
+
+# --------------------------------------------------------------------------- dynamic range
+
+def _bf16(x):
+    return synth.f32_to_bf16_bits(np.asarray(x, dtype=np.float32))
+
+
+def test_token_with_one_huge_channel():
+    # one channel of one token is 1e4 among N(0,1): the per-token power-of-two scale has to keep
+    # both the outlier and the ordinary channels inside the fp16 operands' range
+    n, d_in, d_out, q, g = 96, 512, 256, 3, 128
+    _, X, dY, bits, alpha, _, _ = make_case(900, n, d_in, d_out, q, g)
+    Xf = synth.bf16_bits_to_f32(X)
+    Xf[5, 77] = 1.0e4
+    Xf[40, 300] = -3.0e4
+    X = _bf16(Xf)
+    Xd, _, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    Y = bcq.linear_fwd(Xd, bd, ad, d_in, g).cpu().numpy()
+    assert np.isfinite(Y).all()
+    # per token, since the two outlier tokens dwarf the others
+    for t in (0, 5, 40, 95):
+        assert np.abs(Y[t] - ref[t]).max() <= TOL * np.abs(ref[t]).max()
+    pack = bcq.decode_pack(bd, ad, d_in, g)
+    for nn in (1, 16):
+        refd = ref[:nn * 6:6]
+        Xs = Xd[:nn * 6:6].contiguous()
+        for Yd in (bcq.linear_decode(Xs, bd, ad, d_in, g).cpu().numpy(),
+                   bcq.linear_decode_packed(Xs, pack, d_out, d_in, q, g).cpu().numpy()):
+            for t in range(nn):
+                assert np.abs(Yd[t] - refd[t]).max() <= TOL * np.abs(refd[t]).max()
+
+
+def test_tiny_output_gradients():
+    # dY ~ 1e-6: far below the smallest normal fp16 number unless each token row is rescaled
+    n, d_in, d_out, q, g = 200, 384, 256, 4, 128
+    _, X, dY, bits, alpha, _, _ = make_case(901, n, d_in, d_out, q, g)
+    dY = _bf16(synth.bf16_bits_to_f32(dY) * np.float32(1e-6))
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.bwd_x(dY, bits, alpha, d_in, g)
+    assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g).cpu().numpy(), ref) <= TOL
+    ref = oracle.bwd_alpha(dY, X, bits, d_in, g)
+    assert rel_err(bcq.linear_bwd_alpha(dYd, Xd, bd, d_in, g).cpu().numpy(), ref) <= TOL
+
+
+def test_scales_spread_over_4096x_between_rows_and_groups():
+    # alpha differs by 2^12 between rows and, inside a row, between groups (also: the first groups
+    # of a row are ~1e-6 of the later ones, and the other way round)
+    n, d_in, d_out, q, g = 80, 1024, 256, 3, 128
+    W = synth.weights(d_out, d_in, (100, 902, 0))
+    row_mul = np.float32(2.0) ** -(np.arange(d_out) % 13).astype(np.float32)
+    W = W * row_mul[:, None]
+    W[64:128, :512] *= np.float32(1e-6)     # tiny first four groups
+    W[128:192, 512:] *= np.float32(1e-6)    # tiny last four groups
+    W[192:, 256:384] *= np.float32(4096.0)  # one large group in the middle
+    X = synth.activations(n, d_in, (100, 902, 0), synth.ROLE_X)
+    dY = synth.activations(n, d_out, (100, 902, 0), synth.ROLE_DY)
+    bits, alpha, _, _ = oracle.quantize(W.astype(np.float32), q, g)
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    # decode, column by column: every weight row has its own magnitude and its own scale
+    pack = bcq.decode_pack(bd, ad, d_in, g)
+    for nn in (1, 4, 16):
+        Xs = Xd[:nn].contiguous()
+        for Yd in (bcq.linear_decode(Xs, bd, ad, d_in, g).cpu().numpy(),
+                   bcq.linear_decode_packed(Xs, pack, d_out, d_in, q, g).cpu().numpy()):
+            assert np.isfinite(Yd).all()
+            e = np.abs(Yd - ref[:nn]).max(axis=0) / np.abs(ref).max(axis=0)
+            assert e.max() <= TOL
+    # the prefill kernels scale all weights by one power of two: rows 2^12 below the largest keep
+    # the absolute accuracy of the largest, which the per-tensor metric is about
+    assert rel_err(bcq.linear_fwd(Xd, bd, ad, d_in, g).cpu().numpy(), ref) <= TOL
+    assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g).cpu().numpy(),
+                   oracle.bwd_x(dY, bits, alpha, d_in, g)) <= TOL
+
+
+@pytest.mark.parametrize("n", [1, 2, 4, 7, 16])
+@pytest.mark.parametrize("d_in,d_out,q,g", [
+    (4096, 1536, 3, 128), (1024, 520, 4, 128), (2048, 256, 3, 2048), (1000, 200, 4, 1000),
+    (1600, 336, 4, 128), (320, 384, 2, 96), (256, 128, 1, 32), (2304, 4100, 2, 64),
+])
+def test_decode_packed_matches_oracle(n, d_in, d_out, q, g):
+    _, X, dY, bits, alpha, _, _ = make_case(n + d_out + q, n, d_in, d_out, q, g)
+    Xd, _, bd, ad = _upload(X, dY, bits, alpha)
+    ref = oracle.fwd(X, bits, alpha, d_in, g)
+    pack = bcq.decode_pack(bd, ad, d_in, g)
+    Y = bcq.linear_decode_packed(Xd, pack, d_out, d_in, q, g)
+    Y2 = bcq.linear_decode_packed(Xd, pack, d_out, d_in, q, g)   # the pack's counters are back at zero
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2)
+    assert rel_err(Y.cpu().numpy(), ref) <= TOL
+    bias = synth.bias(d_out, (100, n, 1))
+    Yb = bcq.linear_decode_packed(Xd, pack, d_out, d_in, q, g, bias=torch.from_numpy(bias).cuda(),
+                                  out_dtype=torch.bfloat16)
+    assert rel_err(Yb.float().cpu().numpy(), ref + bias.astype(np.float64)) <= TOL + 2.0 ** -8
+
+
+def test_decode_pack_rejects_more_than_four_planes():
+    assert bcq.lib().bcq_decode_pack_bytes(64, 256, 5, 64) == 0
+    assert bcq.lib().bcq_decode_pack_bytes(64, 256, 4, 64) > 0
+
+
 def test_strided_activations_and_outputs():
     n, d_in, d_out, q, g = 70, 256, 192, 3, 128
     _, X, dY, bits, alpha, _, _ = make_case(3, n, d_in, d_out, q, g)
