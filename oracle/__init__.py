@@ -66,6 +66,10 @@ def _l():
         lib.bcq_ref_bwd_alpha_at.restype = None
         lib.bcq_ref_bwd_alpha_at.argtypes = [i64, i64, i32, i64, i64, vp, i64, vp, i64, vp, dbl,
                                              i64, vp, vp, vp, vp]
+        lib.bcq_ref_lr_linear.restype = dbl
+        lib.bcq_ref_lr_linear.argtypes = [dbl, i64, i64, i64]
+        lib.bcq_ref_adamw.restype = None
+        lib.bcq_ref_adamw.argtypes = [i64, vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, dbl]
         lib.bcq_ref_num_threads.restype = i32
         lib.bcq_ref_num_threads.argtypes = []
         _lib = lib
@@ -234,3 +238,21 @@ def bwd_alpha_at(dY_bf16, X_bf16, bits, d_in: int, g: int, i_idx, j_idx, c_idx,
     _l().bcq_ref_bwd_alpha_at(d_out, d_in, q, g, n, _p(dY), d_out, _p(X), d_in, _p(bits), scale,
                               i_idx.shape[0], _p(i_idx), _p(j_idx), _p(c_idx), _p(out))
     return out
+
+
+def lr_linear(lr0: float, step: int, warmup: int, total: int) -> float:
+    """Learning rate of 0-based step `step`: linear warm-up over `warmup` steps, then linear decay
+    to zero at step `total`."""
+    return float(_l().bcq_ref_lr_linear(lr0, step, warmup, total))
+
+
+def adamw(alpha, grad, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+          eps: float = 1e-8, wd: float = 0.0, grad_scale: float = 1.0):
+    """One AdamW step (1-based `step`) in place on the fp32 arrays alpha, m, v; grad is fp32."""
+    for a in (alpha, m, v):
+        assert a.dtype == np.float32 and a.flags.c_contiguous
+    grad = np.ascontiguousarray(grad, dtype=np.float32)
+    assert alpha.size == grad.size == m.size == v.size
+    _l().bcq_ref_adamw(alpha.size, _p(alpha), _p(grad), _p(m), _p(v), step, lr, beta1, beta2, eps, wd,
+                       grad_scale)
+    return alpha, m, v

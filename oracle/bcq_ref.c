@@ -440,6 +440,43 @@ void bcq_ref_bwd_alpha_at(int64_t d_out, int64_t d_in, int q, int64_t g, int64_t
 }
 
 /* Number of OpenMP threads the loops above will use (1 when built without OpenMP). */
+/* ---------------------------------------------------------------- optimiser -------- */
+
+/* Learning rate of step `step` (0-based) under the linear-decay schedule of Section
+ * "Experimental Setup" ("a linear decay learning rate schedule"; Appendix: "linear-decaying
+ * learning rate scheduler"), with the optional warm-up of the hyper-parameter ablation table:
+ * the rate rises linearly from 0 to lr0 over `warmup` steps, then falls linearly to 0 at step
+ * `total`. */
+double bcq_ref_lr_linear(double lr0, int64_t step, int64_t warmup, int64_t total) {
+    if (step < warmup) return lr0 * (double)step / (double)warmup;
+    if (step >= total) return 0.0;
+    return lr0 * (double)(total - step) / (double)(total - warmup);
+}
+
+/* One AdamW step on the scales (Appendix "Experimental Details": "AdamW optimizer"), i.e. Adam
+ * with decoupled weight decay (Loshchilov & Hutter), t = step (1-based):
+ *     g      = grad_scale * grad            grad_scale = 1/g_L is the paper's Eq. 4 factor
+ *     alpha <- alpha * (1 - lr * wd)
+ *     m     <- beta1 m + (1 - beta1) g ;    v <- beta2 v + (1 - beta2) g^2
+ *     alpha <- alpha - lr * (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+ * alpha, m, v are stored in fp32 (as the trainable state is); the arithmetic of a step is fp64
+ * and each stored value is rounded once. */
+void bcq_ref_adamw(int64_t count, float* alpha, const float* grad, float* m, float* v, int64_t step,
+                   double lr, double beta1, double beta2, double eps, double wd, double grad_scale) {
+    const double bc1 = 1.0 - pow(beta1, (double)step);
+    const double bc2 = 1.0 - pow(beta2, (double)step);
+    for (int64_t e = 0; e < count; ++e) {
+        const double g = grad_scale * (double)grad[e];
+        double a = (double)alpha[e] * (1.0 - lr * wd);
+        const double mm = beta1 * (double)m[e] + (1.0 - beta1) * g;
+        const double vv = beta2 * (double)v[e] + (1.0 - beta2) * g * g;
+        a -= lr * (mm / bc1) / (sqrt(vv / bc2) + eps);
+        alpha[e] = (float)a;
+        m[e] = (float)mm;
+        v[e] = (float)vv;
+    }
+}
+
 #ifdef _OPENMP
 #include <omp.h>
 int bcq_ref_num_threads(void) { return omp_get_max_threads(); }
