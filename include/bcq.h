@@ -214,6 +214,42 @@ bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, int n, const 
                                 uint32_t plane_mask, float scale, int accumulate, float* dalpha,
                                 void* ws, size_t ws_bytes, void* stream);
 
+/* ------------------------------------------------------------------ the AlphaTuning update */
+
+/* Learning rate of 0-based step `step` under the schedule the paper trains with (Section
+ * "Experimental Setup": linear decay; the hyper-parameter ablation also uses a warm-up): linear
+ * rise from 0 to lr0 over warmup_steps (0 = none), then linear decay to 0 at total_steps.  Host
+ * function. */
+float bcq_lr_linear_decay(float lr0, long long step, long long warmup_steps, long long total_steps);
+
+/* One AdamW step (Appendix "Experimental Details": AdamW; decoupled weight decay, bias-corrected
+ * moments) on the trained scales of a whole model in one launch.  alpha, dalpha, m, v are flat
+ * fp32 device arrays with the same indexing: every linear's alpha[q][d_out][G] one after the
+ * other.  The trained elements are `count` elements given by nseg segments -- seg_begin[s] is the
+ * first flat index of segment s, seg_prefix[s] the number of trained elements before it
+ * (seg_prefix[nseg] = count), both int64 DEVICE arrays; a plane of a linear is one segment, so
+ * "alpha_1 of every linear" (what the paper trains) is one segment per linear.  nseg = 0 updates
+ * the contiguous range [0, count).  For element e with gradient g = grad_scale * seg_scale[s] *
+ * dalpha[e] (seg_scale: float device array or NULL = 1; 1/g_L of Eq. 4 goes here when dalpha was
+ * computed with scale 1), t = step (1-based):
+ *     m <- beta1 m + (1 - beta1) g;   v <- beta2 v + (1 - beta2) g^2
+ *     alpha <- alpha (1 - lr weight_decay) - lr (m / (1 - beta1^t)) / (sqrt(v / (1 - beta2^t)) + eps)
+ * in fp32.  Elements outside the segments, and their moments, are not touched. */
+bcq_status bcq_alpha_adamw(long long count, int nseg, const long long* seg_begin, const long long* seg_prefix,
+                           const float* seg_scale, float* alpha, const float* dalpha, float* m, float* v,
+                           long long step, float lr, float beta1, float beta2, float eps, float weight_decay,
+                           float grad_scale, void* stream);
+
+/* The scale-only checkpoint (the paper's per-task checkpoint holds nothing but the trained
+ * alpha): bcq_alpha_pack gathers the segments' elements of the flat array into the compact array
+ * packed[count], in segment order; bcq_alpha_unpack scatters them back.  Layout of a checkpoint =
+ * that compact fp32 array; the segments are a function of the model's shapes and the trained
+ * planes alone. */
+bcq_status bcq_alpha_pack(long long count, int nseg, const long long* seg_begin, const long long* seg_prefix,
+                          const float* alpha_flat, float* packed, void* stream);
+bcq_status bcq_alpha_unpack(long long count, int nseg, const long long* seg_begin, const long long* seg_prefix,
+                            const float* packed, float* alpha_flat, void* stream);
+
 /* ------------------------------------------------------------------ status */
 
 const char* bcq_status_string(int status);

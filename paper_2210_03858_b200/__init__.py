@@ -25,7 +25,8 @@ SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_cou
            "bcq_linear_fwd", "bcq_linear_decode", "bcq_linear_bwd_x", "bcq_linear_bwd_alpha",
            "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag",
            "bcq_kernel_launches", "bcq_linear_decode_noalloc", "bcq_decode_pack_bytes",
-           "bcq_decode_pack", "bcq_linear_decode_packed")
+           "bcq_decode_pack", "bcq_linear_decode_packed", "bcq_lr_linear_decay", "bcq_alpha_adamw",
+           "bcq_alpha_pack", "bcq_alpha_unpack")
 
 
 class BcqError(RuntimeError):
@@ -77,6 +78,15 @@ def lib() -> C.CDLL:
         l.bcq_linear_decode_packed.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_bwd_x.restype = i
         l.bcq_linear_bwd_x.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
+        ll = C.c_longlong
+        l.bcq_lr_linear_decay.restype = f32
+        l.bcq_lr_linear_decay.argtypes = [f32, ll, ll, ll]
+        l.bcq_alpha_adamw.restype = i
+        l.bcq_alpha_adamw.argtypes = [ll, i, vp, vp, vp, vp, vp, vp, vp, ll, f32, f32, f32, f32, f32, f32, vp]
+        l.bcq_alpha_pack.restype = i
+        l.bcq_alpha_pack.argtypes = [ll, i, vp, vp, vp, vp, vp]
+        l.bcq_alpha_unpack.restype = i
+        l.bcq_alpha_unpack.argtypes = [ll, i, vp, vp, vp, vp, vp]
         l.bcq_linear_bwd_alpha.restype = i
         l.bcq_linear_bwd_alpha.argtypes = [i, i, i, i, i, vp, sz, vp, sz, vp, u32, f32, i, vp, vp, sz, vp]
         l.bcq_status_string.restype = C.c_char_p
@@ -291,6 +301,60 @@ def linear_bwd_alpha(dY, X, bits, d_in: int, g: int, plane_mask=None, scale: flo
                                       1 if accumulate else 0, _ptr(out), _ptr(ws), ws_bytes,
                                       _stream()), "bcq_linear_bwd_alpha")
     return out
+
+
+# ---------------------------------------------------------------------------- the update
+
+def lr_linear_decay(lr0: float, step: int, warmup_steps: int, total_steps: int) -> float:
+    return float(lib().bcq_lr_linear_decay(lr0, step, warmup_steps, total_steps))
+
+
+class Segments:
+    """Device-side description of the trained elements of the flat scale arrays: (begin, count)
+    runs -- e.g. AlphaBucket.plane_segments(1) for "alpha_1 of every linear" -- with an optional
+    gradient scale per run (1/g_L of Eq. 4)."""
+
+    def __init__(self, runs, device, scales=None):
+        torch = _torch()
+        self.nseg = len(runs)
+        prefix = [0]
+        for _, c in runs:
+            prefix.append(prefix[-1] + int(c))
+        self.count = prefix[-1]
+        self.begin = torch.tensor([int(b) for b, _ in runs], dtype=torch.int64, device=device)
+        self.prefix = torch.tensor(prefix, dtype=torch.int64, device=device)
+        self.scale = None if scales is None else torch.tensor(list(scales), dtype=torch.float32, device=device)
+
+
+def alpha_adamw(alpha, dalpha, m, v, step: int, lr: float, beta1: float = 0.9, beta2: float = 0.999,
+                eps: float = 1e-8, weight_decay: float = 0.0, grad_scale: float = 1.0, segments: Segments = None):
+    """bcq_alpha_adamw on flat fp32 tensors (in place).  Without segments the whole arrays are updated."""
+    torch = _torch()
+    for t in (alpha, dalpha, m, v):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.numel() == alpha.numel()
+    if segments is None:
+        count, nseg, b, pfx, sc = alpha.numel(), 0, None, None, None
+    else:
+        count, nseg, b, pfx, sc = segments.count, segments.nseg, segments.begin, segments.prefix, segments.scale
+    _check(lib().bcq_alpha_adamw(count, nseg, _ptr(b), _ptr(pfx), _ptr(sc), _ptr(alpha), _ptr(dalpha), _ptr(m),
+                                 _ptr(v), step, lr, beta1, beta2, eps, weight_decay, grad_scale, _stream()),
+           "bcq_alpha_adamw")
+
+
+def alpha_pack(alpha_flat, segments: Segments):
+    """bcq_alpha_pack: the trained scales as one compact fp32 tensor (the per-task checkpoint)."""
+    torch = _torch()
+    out = torch.empty(segments.count, dtype=torch.float32, device=alpha_flat.device)
+    _check(lib().bcq_alpha_pack(segments.count, segments.nseg, _ptr(segments.begin), _ptr(segments.prefix),
+                                _ptr(alpha_flat), _ptr(out), _stream()), "bcq_alpha_pack")
+    return out
+
+
+def alpha_unpack(packed, alpha_flat, segments: Segments):
+    """bcq_alpha_unpack: writes a checkpoint's scales back into the flat array."""
+    assert packed.numel() == segments.count
+    _check(lib().bcq_alpha_unpack(segments.count, segments.nseg, _ptr(segments.begin), _ptr(segments.prefix),
+                                  _ptr(packed), _ptr(alpha_flat), _stream()), "bcq_alpha_unpack")
 
 
 def kernel_launches() -> int:

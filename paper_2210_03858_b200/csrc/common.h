@@ -36,6 +36,21 @@ inline bcq_status check_shape(int d_out, int d_in, int q, int g) {
     return BCQ_OK;
 }
 
+// Number of SMs of the current device (148 on a B200; that value is also the answer when no device
+// can be asked, e.g. for size queries on a machine without a GPU).
+inline int sm_count() {
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            return 148;  // not cached, so a later call with a device present asks again
+    }
+    return cached;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

@@ -245,7 +245,7 @@ cudaError_t launch_quantize(const QuantParams& p, cudaStream_t stream) {
     constexpr int TEAMS = (TW == 1) ? 4 : 1;
     const int threads = (TW == 1) ? 128 : TW * 32;
     long long blocks = (p.items + TEAMS - 1) / TEAMS;
-    const long long cap = 148LL * 64;  // grid-stride beyond this
+    const long long cap = (long long)bcq::sm_count() * 64;  // grid-stride beyond this
     if (blocks > cap) blocks = cap;
     if (p.alt_iters > 0)
         quantize_kernel<EPT, TW, true><<<(unsigned)blocks, threads, 0, stream>>>(p);
