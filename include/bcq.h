@@ -128,6 +128,26 @@ bcq_status bcq_linear_fwd(int d_out, int d_in, int q, int g, int n, const void* 
                           const uint32_t* bits, const float* alpha, const float* bias, void* Y,
                           size_t ldy, int y_dtype, void* ws, size_t ws_bytes, void* stream);
 
+/* Planes prepared once.  AlphaTuning freezes B after quantization and trains only alpha, so the
+ * regrouping of the planes that bcq_linear_fwd / bcq_linear_bwd_x do on every call can be done once
+ * per layer: bcq_prepare_planes writes, for op = BCQ_OP_FWD or BCQ_OP_BWD_X, the planes in the
+ * chunk order of that kernel with every weight's level index already in the form the expansion
+ * consumes (q <= 4; q > 4 gives BCQ_ERR_UNSUPPORTED and keeps using the calls above).  The buffer
+ * is bcq_prepared_bytes() bytes (0 if unsupported; about bcq_bits_bytes(), more for q = 1 or 2,
+ * which are stored like q = 3), 16-byte aligned, caller-owned, and read-only for the *_prepared
+ * calls, which take it in place of `bits` and otherwise behave exactly like bcq_linear_fwd /
+ * bcq_linear_bwd_x (same results bit for bit, same workspace sizes).  alpha stays an argument of
+ * every call: it changes with every optimiser step. */
+size_t bcq_prepared_bytes(int op, int d_out, int d_in, int q, int g);
+bcq_status bcq_prepare_planes(int op, int d_out, int d_in, int q, int g, const uint32_t* bits,
+                              void* prepared, size_t prepared_bytes, void* stream);
+bcq_status bcq_linear_fwd_prepared(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                                   const void* prepared, const float* alpha, const float* bias, void* Y,
+                                   size_t ldy, int y_dtype, void* ws, size_t ws_bytes, void* stream);
+bcq_status bcq_linear_bwd_x_prepared(int d_out, int d_in, int q, int g, int n, const void* dY, size_t lddy,
+                                     const void* prepared, const float* alpha, void* dX, size_t lddx,
+                                     int dx_dtype, void* ws, size_t ws_bytes, void* stream);
+
 /* Same computation for the decode regime, 1 <= n <= 16 tokens, where the cost is streaming
  * the packed planes from memory once (Section "Inference Speed").  Workspace op is
  * BCQ_OP_DECODE.  n > 16 gives BCQ_ERR_SHAPE. */

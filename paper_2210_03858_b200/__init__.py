@@ -26,7 +26,8 @@ SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_cou
            "bcq_status_string", "bcq_last_cuda_error", "bcq_device_timeout_flag",
            "bcq_kernel_launches", "bcq_linear_decode_noalloc", "bcq_decode_pack_bytes",
            "bcq_decode_pack", "bcq_linear_decode_packed", "bcq_lr_linear_decay", "bcq_alpha_adamw",
-           "bcq_alpha_pack", "bcq_alpha_unpack")
+           "bcq_alpha_pack", "bcq_alpha_unpack", "bcq_prepared_bytes", "bcq_prepare_planes",
+           "bcq_linear_fwd_prepared", "bcq_linear_bwd_x_prepared")
 
 
 class BcqError(RuntimeError):
@@ -78,6 +79,14 @@ def lib() -> C.CDLL:
         l.bcq_linear_decode_packed.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
         l.bcq_linear_bwd_x.restype = i
         l.bcq_linear_bwd_x.argtypes = [i, i, i, i, i, vp, sz, vp, vp, vp, sz, i, vp, sz, vp]
+        l.bcq_prepared_bytes.restype = sz
+        l.bcq_prepared_bytes.argtypes = [i, i, i, i, i]
+        l.bcq_prepare_planes.restype = i
+        l.bcq_prepare_planes.argtypes = [i, i, i, i, i, vp, vp, sz, vp]
+        l.bcq_linear_fwd_prepared.restype = i
+        l.bcq_linear_fwd_prepared.argtypes = l.bcq_linear_fwd.argtypes
+        l.bcq_linear_bwd_x_prepared.restype = i
+        l.bcq_linear_bwd_x_prepared.argtypes = l.bcq_linear_bwd_x.argtypes
         ll = C.c_longlong
         l.bcq_lr_linear_decay.restype = f32
         l.bcq_lr_linear_decay.argtypes = [f32, ll, ll, ll]
@@ -193,9 +202,36 @@ def dequantize(bits, alpha, d_in: int, g: int):
     return W_hat
 
 
+class PreparedPlanes:
+    """The frozen planes of one layer as written by bcq_prepare_planes for one operation."""
+
+    def __init__(self, op, buf, q, d_out, d_in, g):
+        self.op, self.buf, self.q, self.d_out, self.d_in, self.g = op, buf, q, d_out, d_in, g
+        self.shape = (q, d_out, pitch_words(d_in))   # shape of the canonical planes it stands for
+
+    def data_ptr(self):
+        return self.buf.data_ptr()
+
+
+def prepare_planes(op: int, bits, d_in: int, g: int) -> PreparedPlanes:
+    """bcq_prepare_planes for op = OP_FWD or OP_BWD_X (q <= 4)."""
+    torch = _torch()
+    q, d_out, _ = bits.shape
+    nbytes = lib().bcq_prepared_bytes(op, d_out, d_in, q, g)
+    if nbytes == 0:
+        raise BcqError(-4, "bcq_prepared_bytes")
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=bits.device)
+    _check(lib().bcq_prepare_planes(op, d_out, d_in, q, g, _ptr(bits), _ptr(buf), nbytes, _stream()),
+           "bcq_prepare_planes")
+    return PreparedPlanes(op, buf, q, d_out, d_in, g)
+
+
 def _fwd(fn, op, name, X, bits, alpha, d_in, g, bias, out, out_dtype, ws):
     torch = _torch()
     assert X.is_cuda and X.dtype == torch.bfloat16 and X.dim() == 2 and X.stride(1) == 1
+    if isinstance(bits, PreparedPlanes):
+        assert bits.op == OP_FWD and op == OP_FWD
+        fn, name = lib().bcq_linear_fwd_prepared, "bcq_linear_fwd_prepared"
     q, d_out, _ = bits.shape
     n = X.shape[0]
     if out is None:
@@ -276,9 +312,12 @@ def linear_bwd_x(dY, bits, alpha, d_in: int, g: int, out=None, out_dtype=None, w
     if out is None:
         out = torch.empty((n, d_in), dtype=out_dtype or torch.float32, device=dY.device)
     ws, ws_bytes = _ws(OP_BWD_X, d_out, d_in, q, g, n, ws, dY.device)
-    _check(lib().bcq_linear_bwd_x(d_out, d_in, q, g, n, _ptr(dY), dY.stride(0), _ptr(bits),
-                                  _ptr(alpha), _ptr(out), out.stride(0), _dtype_code(out),
-                                  _ptr(ws), ws_bytes, _stream()), "bcq_linear_bwd_x")
+    fn, name = lib().bcq_linear_bwd_x, "bcq_linear_bwd_x"
+    if isinstance(bits, PreparedPlanes):
+        assert bits.op == OP_BWD_X
+        fn, name = lib().bcq_linear_bwd_x_prepared, "bcq_linear_bwd_x_prepared"
+    _check(fn(d_out, d_in, q, g, n, _ptr(dY), dY.stride(0), _ptr(bits), _ptr(alpha), _ptr(out),
+              out.stride(0), _dtype_code(out), _ptr(ws), ws_bytes, _stream()), name)
     return out
 
 

@@ -163,27 +163,16 @@ __global__ void pack_codes_kernel(int d_out, int pitch, int q, int m_tiles, int 
     const bool valid = (j < d_out) && (word < pitch);
     for (int i = 0; i < q; ++i)
         if (valid) w[i] = __ldg(bits + ((long long)i * d_out + j) * pitch + word);
-    uint32_t S[4] = {0u, 0u, 0u, 0u};
-    for (int e = 0; e < 32; ++e) {
-        uint32_t code = 0u;
-        for (int i = 0; i < 3 && i < q; ++i) code |= ((w[i] >> e) & 1u) << i;
-        if (q == 4 && !((w[3] >> e) & 1u)) code = (~code & 7u) | 8u;
-        S[e >> 3] |= code << (4 * (e & 7));
-    }
+    uint32_t S[4];
+    selectors_from_planes(w, q, S);
     if (!valid)
         for (int r = 0; r < 4; ++r) S[r] = 0u;
     uint32_t* dst = codes + idx * q;  // [unit][quarter][row][q words]
-    if (q == 4) {
-        for (int r = 0; r < 4; ++r) dst[r] = S[r];
-    } else if (q == 3) {
-        // bit 3 of every nibble of the first three words carries selector word 3:
-        // nibble e of word v gets bit v of nibble e of S[3]
-        for (int v = 0; v < 3; ++v) dst[v] = S[v] | (((S[3] >> v) & 0x11111111u) << 3);
-    } else if (q == 2) {
-        dst[0] = S[0] | (S[1] << 2);
-        dst[1] = S[2] | (S[3] << 2);
-    } else {
-        dst[0] = S[0] | (S[1] << 1) | (S[2] << 2) | (S[3] << 3);
+    switch (q) {
+        case 4: pack_selectors<4>(S, dst); break;
+        case 3: pack_selectors<3>(S, dst); break;
+        case 2: pack_selectors<2>(S, dst); break;
+        default: pack_selectors<1>(S, dst); break;
     }
 }
 
@@ -217,66 +206,6 @@ __host__ __device__ inline int range_begin(int c, int per, int rem) { return c *
 __host__ __device__ inline int unit_owner(int u, int per, int rem) {
     const int big = rem * (per + 1);
     return u < big ? u / (per + 1) : rem + (u - big) / per;
-}
-
-template <int Q>
-__device__ __forceinline__ void load_codes(uint32_t addr, uint32_t (&v)[Q]) {
-    if constexpr (Q == 4) {
-        asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3])
-                     : "r"(addr) : "memory");
-    } else if constexpr (Q == 2) {
-        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v[0]), "=r"(v[1]) : "r"(addr) : "memory");
-    } else {
-#pragma unroll
-        for (int i = 0; i < Q; ++i) v[i] = ptx::ld_shared_u32(addr + 4 * i);
-    }
-}
-
-// The four selector words of 32 weights from the q stored words (see pack_codes_kernel).
-template <int Q>
-__device__ __forceinline__ void selectors(const uint32_t (&v)[Q], uint32_t (&S)[4]) {
-    constexpr uint32_t M = 0x11111111u;
-    if constexpr (Q == 4) {
-#pragma unroll
-        for (int r = 0; r < 4; ++r) S[r] = v[r];
-    } else if constexpr (Q == 3) {
-#pragma unroll
-        for (int r = 0; r < 3; ++r) S[r] = v[r] & 0x77777777u;
-        S[3] = (__umulhi(v[0], 1u << 29) & M) | (__umulhi(v[1], 1u << 30) & (M << 1)) | (__umulhi(v[2], 1u << 31) & (M << 2));
-    } else if constexpr (Q == 2) {
-        S[0] = v[0] & 0x33333333u;
-        S[1] = (v[0] >> 2) & 0x33333333u;
-        S[2] = v[1] & 0x33333333u;
-        S[3] = (v[1] >> 2) & 0x33333333u;
-    } else {
-#pragma unroll
-        for (int r = 0; r < 4; ++r) S[r] = (v[0] >> r) & M;
-    }
-}
-
-// 32 weights of one row: selector word r gives the eight fp16 values of 16-byte chunk chunk0 + r
-// of the row's 128-byte line (swizzle key lx), in natural k order.
-template <int Q>
-__device__ __forceinline__ void expand32_codes(const uint32_t (&S)[4], const Lut& t, uint32_t line, uint32_t lx,
-                                               uint32_t chunk0) {
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        // (shifts written as multiplications run on the multiply-add pipe; the logic pipe, which does
-        // the PRMTs, is the one that paces this loop)
-        const uint32_t s = (Q == 4) ? (S[r] & 0x77777777u) : S[r];
-        const uint32_t sh = __umulhi(s, 1u << 16);
-        const uint32_t lbl = prmt(t.tl0, t.tl1, s), lbh = prmt(t.tl0, t.tl1, sh);
-        uint32_t hbl = prmt(t.th0, t.th1, s), hbh = prmt(t.th0, t.th1, sh);
-        if (Q == 4) {
-            // bit 3 of nibble e = "negate": replicate it over byte e (PRMT's sign mode reads the most
-            // significant bit of a byte; shifting by 4 brings the even nibbles' flags there)
-            const uint32_t fa = S[r] * 16u;
-            hbl ^= prmt(fa, S[r], 0xD9C8u) & 0x80808080u;
-            hbh ^= prmt(fa, S[r], 0xFBEAu) & 0x80808080u;
-        }
-        ptx::st_shared_v4(line + (((chunk0 + r) ^ lx) << 4), prmt(lbl, hbl, 0x5140u), prmt(lbl, hbl, 0x7362u),
-                          prmt(lbh, hbh, 0x5140u), prmt(lbh, hbh, 0x7362u));
-    }
 }
 
 __device__ __forceinline__ uint32_t max_mag_bf16x8_masked(const uint4& x, int k0, int K) {
@@ -567,14 +496,16 @@ decode_packed_kernel(const DecPackedParams p) {
             Lut t;
             asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(t.tl0), "=r"(t.tl1), "=r"(t.th0), "=r"(t.th1)
                          : "r"(chunk + table_off) : "memory");
-            // the chunk is in registers: hand it back, then wait for the operand slot
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(wempty + 8 * r);
             ok = wait_bar(ctl.empty + 8 * a, aph ^ 1u, ctl, 38);
             if (!ok) return;
             uint32_t S[4];
             selectors<Q>(v, S);
             expand32_codes<Q>(S, t, a_base + (uint32_t)a * kDpABytes + line_off, lx, chunk0);
+            // the chunk goes back to the producer only now that what was loaded from it has been
+            // consumed: a load that has merely been issued may still be reading shared memory when
+            // the next bulk copy (another proxy) overwrites the slot
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(wempty + 8 * r);
             if (++r == RING) { r = 0; rph ^= 1u; }
         };
         // B operand of the step whose activations are in xv, then the slot is complete

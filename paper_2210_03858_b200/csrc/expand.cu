@@ -154,6 +154,13 @@ struct NumWords {
     static constexpr int value = (QM == QM_GENERIC) ? BCQ_MAX_Q : 4;
 };
 
+// Stored words per 32 weights when the planes are kept as selector codes (q <= 4): the q = 4
+// packing for four planes, the q = 3 packing for one to three (missing planes read as index bits 0).
+template <int QM>
+struct CodeWords {
+    static constexpr int value = (QM == QM_LUT4) ? 4 : 3;
+};
+
 // The scales of one (row, group), already multiplied by the weight scale; loaded ahead of use.
 template <int QM>
 struct AlphaSet {
@@ -434,6 +441,37 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
     } else {
         for (int v = lane; v < nvec; v += 32) dst[v] = scale_to_fp16x8(__ldg(src + v), v * 8, p.K, scale);
     }
+}
+
+// Selector codes of the planes (q <= 4) in the chunk order of the GEMM kernel; one thread per (row,
+// 32-weight block).  The planes are frozen, so this runs once per layer (bcq_prepare_planes); a call
+// that is not given prepared planes runs it into its workspace.
+//   forward  codes [m_tile][kb][128 rows][2 halves][NW words]    NW = CodeWords
+//   dX       codes [u][jb][64 rows][4 quarters][NW words]
+// Rows past d_out and blocks past the row pitch are written as zeros (their levels are zero or
+// meet zero activations).
+template <int NW>
+__global__ void __launch_bounds__(256) code_planes_kernel(int mode, int d_out, int pitch, int q, int rows_padded,
+                                                           int words_padded, int num_kb, const uint32_t* __restrict__ bits,
+                                                           uint32_t* __restrict__ codes) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)rows_padded * words_padded) return;
+    const int wd = (int)(idx % words_padded);
+    const int j = (int)(idx / words_padded);
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+    const bool valid = (j < d_out) && (wd < pitch);
+    for (int i = 0; i < q; ++i)
+        if (valid) w[i] = __ldg(bits + ((long long)i * d_out + j) * pitch + wd);
+    uint32_t S[4];
+    selectors_from_planes(w, q, S);
+    if (!valid)
+        for (int r = 0; r < 4; ++r) S[r] = 0u;
+    long long o;
+    if (mode == MODE_FWD)
+        o = ((((long long)(j >> 7) * num_kb + (wd >> 1)) * 128 + (j & 127)) * 2 + (wd & 1)) * NW;
+    else
+        o = ((((long long)(wd >> 2) * num_kb + (j >> 6)) * 64 + (j & 63)) * 4 + (wd & 3)) * NW;
+    pack_selectors<NW>(S, codes + o);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -785,7 +823,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // which of the stage's alpha parts covers this thread's 32 k
         const int apart = (MODE == MODE_FWD) ? (p.alpha_parts == 2 ? part : 0)
                                              : (p.alpha_parts == 4 ? part : (p.alpha_parts == 2 ? (part >> 1) : 0));
-        const uint32_t w_off = (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4
+        const uint32_t w_off = (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4 (q > 4: plane words)
+        constexpr int NWC = CodeWords<QM>::value;
+        const uint32_t c_off = (uint32_t)((row * kUnit + part) * NWC) * 4;               // q <= 4: selector codes
         const uint32_t a_off = p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
 
         Lut lut = {0u, 0u, 0u, 0u};
@@ -816,16 +856,23 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 const uint32_t stage = smem_base + s * kStageBytes;
                 const uint32_t aux = aux_base + as * kAuxBytes;
                 uint32_t w[NW];
+                uint32_t cv[NWC];
+                if (QM == QM_GENERIC) {
 #pragma unroll
-                for (int i = 0; i < NW; ++i)
-                    w[i] = (i < p.q) ? ptx::ld_shared_u32(aux + w_off + i * (kRows * kUnit * 4)) : 0u;
-                // everything this warp needs from the chunk is in registers: hand the aux slot back,
-                // then wait until the UMMAs that read the operand slot's previous contents are done
-                auto release_and_acquire = [&]() {
+                    for (int i = 0; i < NW; ++i)
+                        w[i] = (i < p.q) ? ptx::ld_shared_u32(aux + w_off + i * (kRows * kUnit * 4)) : 0u;
+                } else {
+                    load_codes<NWC>(aux + c_off, cv);
+                }
+                // The aux slot is handed back only after the expansion below has consumed what was
+                // loaded from it: a load that has merely been issued may still be reading shared
+                // memory when the producer's next bulk copy (another proxy) overwrites the slot.
+                auto release_aux = [&]() {
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(wempty + 8 * as);
-                    return wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9);
                 };
+                // until the UMMAs that read the operand slot's previous contents are done
+                auto acquire_slot = [&]() { return wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9); };
                 if (QM == QM_GENERIC) {
                     float a8[BCQ_MAX_Q];
                     uint32_t w8[BCQ_MAX_Q];
@@ -834,12 +881,13 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                         a8[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
                         w8[i] = w[i % NW];
                     }
-                    ok = release_and_acquire();
+                    ok = acquire_slot();
                     if (!ok) break;
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0);
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
                     expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0 + 2);
+                    release_aux();
                 } else {
                     const int key = cw;
                     if (MODE == MODE_BWDX || key != lut_key) {  // dX: every stage brings other rows
@@ -850,9 +898,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                         lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
                         lut_key = key;
                     }
-                    ok = release_and_acquire();
+                    ok = acquire_slot();
                     if (!ok) break;
-                    expand32_lut<QM == QM_LUT4>(w[0], w[1], w[2], w[3], lut, stage + line_off, lx, chunk0);
+                    uint32_t S[4];
+                    selectors<NWC>(cv, S);
+                    expand32_codes<NWC>(S, lut, stage + line_off, lx, chunk0);
+                    release_aux();
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
@@ -1336,6 +1387,7 @@ struct ExpandPlan {
     int TN, splits, kb_per_split, num_kb, m_tiles, n_tiles;
     int stages, aux_slots, epi_bufs, alpha_parts;
     uint32_t bits_bytes, alpha_bytes;
+    size_t planes_bytes;                                                 // the regrouped planes (codes for q <= 4)
     size_t smem;                                                         // dynamic shared memory of the GEMM kernel
     size_t off_tok, off_act, off_alpha, off_bits, off_partial, total;  // workspace layout (bytes)
     int ld_act;                                                          // pitch of the fp16 activations (elements)
@@ -1379,7 +1431,7 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     const int kspan = (mode == MODE_FWD) ? 64 : 128;
     pl.alpha_parts = (g % kspan == 0) ? 1 : ((g % (kspan / 2) == 0) ? 2 : 4);
     if (mode == MODE_FWD && pl.alpha_parts == 4) pl.alpha_parts = 2;  // g % 32 == 0 always holds
-    pl.bits_bytes = (uint32_t)q * 1024u;
+    pl.bits_bytes = (q <= 3 ? 3u : (uint32_t)q) * 1024u;  // q <= 4: selector codes (3 or 4 words per 32 weights)
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
     const size_t ab_bytes = kABytes + (size_t)tn * kBlockK * 2;
     const size_t aux_bytes = pl.bits_bytes + (size_t)pl.alpha_parts * pl.alpha_bytes;
@@ -1413,7 +1465,8 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     pl.off_act = align_up(pl.off_tok + (size_t)n * sizeof(float), 128);
     pl.off_alpha = align_up(pl.off_act + (size_t)n * pl.ld_act * 2, 128);
     pl.off_bits = align_up(pl.off_alpha + blocks_alpha * pl.alpha_bytes, 128);
-    pl.off_partial = align_up(pl.off_bits + chunks_bits * pl.bits_bytes, 128);
+    pl.planes_bytes = chunks_bits * pl.bits_bytes;
+    pl.off_partial = align_up(pl.off_bits + pl.planes_bytes, 128);
     pl.total = pl.off_partial + (pl.splits > 1 ? (size_t)pl.splits * n * Mdim * sizeof(float) : 0);
     return pl;
 }
@@ -1465,10 +1518,30 @@ bcq_status launch_expand_q(const CUtensorMap& tm, const CUtensorMap& tmo, const 
 }
 
 // act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).
+// Writes the selector codes of the planes (q <= 4) in the chunk order of mode `mode`.
+bcq_status launch_code_planes(int mode, int d_out, int d_in, int q, const ExpandPlan& pl, const uint32_t* bits,
+                              uint32_t* codes, cudaStream_t s) {
+    const int pitch = (int)bcq_pitch_words(d_in);
+    const int rows_padded = (mode == MODE_FWD) ? pl.m_tiles * 128 : pl.num_kb * 64;
+    const int words_padded = (mode == MODE_FWD) ? pl.num_kb * 2 : pl.m_tiles * 4;
+    const long long total = (long long)rows_padded * words_padded;
+    const unsigned grid = (unsigned)((total + 255) / 256);
+    if (q == 4)
+        code_planes_kernel<4><<<grid, 256, 0, s>>>(mode, d_out, pitch, q, rows_padded, words_padded, pl.num_kb, bits, codes);
+    else
+        code_planes_kernel<3><<<grid, 256, 0, s>>>(mode, d_out, pitch, q, rows_padded, words_padded, pl.num_kb, bits, codes);
+    bcq::count_launch();
+    BCQ_CUDA_TRY(cudaGetLastError());
+    return BCQ_OK;
+}
+
+// act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).  `prepared`: the
+// planes as written by bcq_prepare_planes for this mode, or null (then `bits` is regrouped into
+// the workspace by this call).
 template <int MODE>
 bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act, size_t ldact,
-                      const uint32_t* bits, const float* alpha, const float* bias, void* out, size_t ldo,
-                      int out_dtype, void* ws, size_t ws_bytes, void* stream) {
+                      const uint32_t* bits, const void* prepared, const float* alpha, const float* bias, void* out,
+                      size_t ldo, int out_dtype, void* ws, size_t ws_bytes, void* stream) {
     const int Mdim = (MODE == MODE_FWD) ? d_out : d_in;
     const int Kdim = (MODE == MODE_FWD) ? d_in : d_out;
     const ExpandPlan pl = plan_expand(MODE, d_out, d_in, q, g, n);
@@ -1500,11 +1573,15 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     pp.row_tiles = ceil_div(d_out, 128);
     pp.bits_cblk = ceil_div(pitch, 32);
     pp.alpha_cblk = ceil_div(pp.G, 32);
-    pp.bits_blocks = q * pp.row_tiles * pp.bits_cblk;
+    const bool coded = q <= 4;  // selector codes (written once, or by the launch below); q > 4: plane words
+    pp.bits_blocks = coded ? 0 : q * pp.row_tiles * pp.bits_cblk;
     const int alpha_tr_blocks = q * pp.row_tiles * pp.alpha_cblk;
     pp.bits = bits;
     pp.alpha_t = reinterpret_cast<float*>(wsb + pl.off_alpha);
     pp.bits_t = reinterpret_cast<uint32_t*>(wsb + pl.off_bits);
+    if (coded && prepared == nullptr) {
+        if ((st = launch_code_planes(MODE, d_out, d_in, q, pl, bits, pp.bits_t, s)) != BCQ_OK) return st;
+    }
     const int tok_blocks = ceil_div(n, kPrepTokensPerBlock);
     pp.act_blocks = tok_blocks;
     const unsigned pgrid = (unsigned)(tok_blocks + ablocks + pp.bits_blocks + alpha_tr_blocks);
@@ -1525,7 +1602,8 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
     p.stages = pl.stages; p.aux_slots = pl.aux_slots; p.epi_bufs = pl.epi_bufs; p.bits_bytes = pl.bits_bytes;
     p.alpha_bytes = pl.alpha_bytes; p.alpha_parts = pl.alpha_parts;
-    p.bits_t = pp.bits_t; p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
+    p.bits_t = (coded && prepared != nullptr) ? reinterpret_cast<const uint32_t*>(prepared) : pp.bits_t;
+    p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
     // bf16 output with an aligned base and pitch and no K split goes out through TMA stores
@@ -1619,8 +1697,8 @@ bcq_status fwd_common(int decode, int d_out, int d_in, int q, int g, int n, cons
     if (!aligned16(bits)) return BCQ_ERR_ALIGN;
     if (decode)
         return run_decode(d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes, stream);
-    return run_expand<MODE_FWD>(d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes,
-                                stream);
+    return run_expand<MODE_FWD>(d_out, d_in, q, g, n, X, ldx, bits, nullptr, alpha, bias, Y, ldy, y_dtype, ws,
+                                ws_bytes, stream);
 }
 
 }  // namespace
@@ -1720,6 +1798,69 @@ extern "C" bcq_status bcq_linear_bwd_x(int d_out, int d_in, int q, int g, int n,
     if (lddx < (size_t)d_in) return BCQ_ERR_SHAPE;
     if (dx_dtype != BCQ_F32 && dx_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
     if (!aligned16(bits)) return BCQ_ERR_ALIGN;
-    return run_expand<MODE_BWDX>(d_out, d_in, q, g, n, dY, lddy, bits, alpha, nullptr, dX, lddx, dx_dtype, ws,
-                                 ws_bytes, stream);
+    return run_expand<MODE_BWDX>(d_out, d_in, q, g, n, dY, lddy, bits, nullptr, alpha, nullptr, dX, lddx, dx_dtype,
+                                 ws, ws_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------------
+// planes prepared once (B is frozen)
+// ------------------------------------------------------------------------------------------
+
+namespace {
+bcq_status check_prepared(int op, int d_out, int d_in, int q, int g) {
+    bcq_status st = check_shape(d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (op != BCQ_OP_FWD && op != BCQ_OP_BWD_X) return BCQ_ERR_SHAPE;
+    if (q > 4) return BCQ_ERR_UNSUPPORTED;
+    return BCQ_OK;
+}
+}  // namespace
+
+extern "C" size_t bcq_prepared_bytes(int op, int d_out, int d_in, int q, int g) {
+    if (check_prepared(op, d_out, d_in, q, g) != BCQ_OK) return 0;
+    return plan_expand(op == BCQ_OP_FWD ? MODE_FWD : MODE_BWDX, d_out, d_in, q, g, 256).planes_bytes;
+}
+
+extern "C" bcq_status bcq_prepare_planes(int op, int d_out, int d_in, int q, int g, const uint32_t* bits,
+                                         void* prepared, size_t prepared_bytes, void* stream) {
+    bcq_status st = check_prepared(op, d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (!bits || !prepared) return BCQ_ERR_NULL;
+    if (!aligned16(bits) || !aligned16(prepared)) return BCQ_ERR_ALIGN;
+    const int mode = (op == BCQ_OP_FWD) ? MODE_FWD : MODE_BWDX;
+    const ExpandPlan pl = plan_expand(mode, d_out, d_in, q, g, 256);
+    if (prepared_bytes < pl.planes_bytes) return BCQ_ERR_WORKSPACE;
+    return launch_code_planes(mode, d_out, d_in, q, pl, bits, reinterpret_cast<uint32_t*>(prepared),
+                              (cudaStream_t)stream);
+}
+
+extern "C" bcq_status bcq_linear_fwd_prepared(int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                                              const void* prepared, const float* alpha, const float* bias,
+                                              void* Y, size_t ldy, int y_dtype, void* ws, size_t ws_bytes,
+                                              void* stream) {
+    bcq_status st = check_prepared(BCQ_OP_FWD, d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1) return BCQ_ERR_SHAPE;
+    if (!prepared || !alpha || !Y) return BCQ_ERR_NULL;
+    if ((st = check_act(X, ldx, d_in)) != BCQ_OK) return st;
+    if (ldy < (size_t)d_out) return BCQ_ERR_SHAPE;
+    if (y_dtype != BCQ_F32 && y_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
+    if (!aligned16(prepared)) return BCQ_ERR_ALIGN;
+    return run_expand<MODE_FWD>(d_out, d_in, q, g, n, X, ldx, nullptr, prepared, alpha, bias, Y, ldy, y_dtype, ws,
+                                ws_bytes, stream);
+}
+
+extern "C" bcq_status bcq_linear_bwd_x_prepared(int d_out, int d_in, int q, int g, int n, const void* dY,
+                                                size_t lddy, const void* prepared, const float* alpha, void* dX,
+                                                size_t lddx, int dx_dtype, void* ws, size_t ws_bytes, void* stream) {
+    bcq_status st = check_prepared(BCQ_OP_BWD_X, d_out, d_in, q, g);
+    if (st != BCQ_OK) return st;
+    if (n < 1) return BCQ_ERR_SHAPE;
+    if (!prepared || !alpha || !dX) return BCQ_ERR_NULL;
+    if ((st = check_act(dY, lddy, d_out)) != BCQ_OK) return st;
+    if (lddx < (size_t)d_in) return BCQ_ERR_SHAPE;
+    if (dx_dtype != BCQ_F32 && dx_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
+    if (!aligned16(prepared)) return BCQ_ERR_ALIGN;
+    return run_expand<MODE_BWDX>(d_out, d_in, q, g, n, dY, lddy, nullptr, prepared, alpha, nullptr, dX, lddx,
+                                 dx_dtype, ws, ws_bytes, stream);
 }

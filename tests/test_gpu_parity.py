@@ -216,6 +216,32 @@ def test_decode_matches_oracle(n, d_in, d_out, q, g):
     assert rel_err(Y.cpu().numpy(), ref) <= TOL
 
 
+@pytest.mark.parametrize("n,d_in,d_out,q,g", [c for c in LINEAR_CASES if c[3] <= 4] + [(200, 640, 304, 2, 128),
+                                                                                       (300, 1600, 4800, 4, 128)])
+def test_prepared_planes_give_the_same_results(n, d_in, d_out, q, g):
+    # B is frozen: the planes regrouped once must give, bit for bit, what the per-call regrouping gives
+    _, X, dY, bits, alpha, _, _ = make_case(n, n, d_in, d_out, q, g)
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    pf = bcq.prepare_planes(bcq.OP_FWD, bd, d_in, g)
+    px = bcq.prepare_planes(bcq.OP_BWD_X, bd, d_in, g)
+    for dt in (torch.float32, torch.bfloat16):
+        assert torch.equal(bcq.linear_fwd(Xd, pf, ad, d_in, g, out_dtype=dt), bcq.linear_fwd(Xd, bd, ad, d_in, g, out_dtype=dt))
+        assert torch.equal(bcq.linear_bwd_x(dYd, px, ad, d_in, g, out_dtype=dt),
+                           bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=dt))
+    assert rel_err(bcq.linear_fwd(Xd, pf, ad, d_in, g).cpu().numpy(), oracle.fwd(X, bits, alpha, d_in, g)) <= TOL
+    assert rel_err(bcq.linear_bwd_x(dYd, px, ad, d_in, g).cpu().numpy(), oracle.bwd_x(dY, bits, alpha, d_in, g)) <= TOL
+    # alpha may change between calls (it is what AlphaTuning trains); the prepared planes stay valid
+    ad2 = ad * 1.25
+    ref2 = oracle.fwd(X, bits, (alpha * np.float32(1.25)).astype(np.float32), d_in, g)
+    assert rel_err(bcq.linear_fwd(Xd, pf, ad2, d_in, g).cpu().numpy(), ref2) <= TOL
+
+
+def test_prepared_planes_need_at_most_four_planes():
+    assert bcq.lib().bcq_prepared_bytes(bcq.OP_FWD, 64, 256, 5, 64) == 0
+    assert bcq.lib().bcq_prepared_bytes(bcq.OP_BWD_X, 64, 256, 4, 64) > 0
+    assert bcq.lib().bcq_prepared_bytes(bcq.OP_DECODE, 64, 256, 4, 64) == 0
+
+
 # --------------------------------------------------------------------------- tile-schedule corners
 
 @pytest.mark.parametrize("n", [1, 17, 31, 32])
