@@ -1,4 +1,8 @@
 // Host-only entry points: size helpers of the container format, status strings, error state.
+#include <map>
+#include <mutex>
+#include <utility>
+
 #include "gemm_common.cuh"
 
 namespace bcq {
@@ -6,6 +10,20 @@ static thread_local int t_last_cuda_error = 0;
 static thread_local unsigned long long t_launches = 0;
 void set_last_cuda_error(int e) { t_last_cuda_error = e; }
 void count_launch() { ++t_launches; }
+
+bcq_status ensure_dynamic_smem_impl(const void* kern, size_t bytes) {
+    static std::mutex lock;
+    static std::map<std::pair<const void*, int>, size_t> configured;  // (kernel, device) -> bytes granted
+    int dev = 0;
+    BCQ_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> guard(lock);
+    size_t& have = configured[std::make_pair(kern, dev)];
+    if (have < bytes) {
+        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+        have = bytes;
+    }
+    return BCQ_OK;
+}
 }  // namespace bcq
 
 extern "C" size_t bcq_pitch_words(int d_in) {

@@ -21,6 +21,7 @@ struct DalphaParams {
     int num_kb;          // K blocks of 64 tokens
     int kb_per_split;
     int splits;
+    int m_tiles, n_tiles;
     int n_subtiles;      // column sub-tiles of width TN/2 over d_in
     int slots;           // partial slots per sub-tile
     uint32_t plane_mask;
@@ -33,6 +34,11 @@ struct DalphaParams {
 // dalpha: D[j, k] = sum_t dY[t, j] X[t, k], sign-weighted group sums in the epilogue
 // ------------------------------------------------------------------------------------------
 
+// Persistent: every CTA walks over (row tile, column tile, token split) tiles; two accumulators
+// in tensor memory, so the sign-and-sum epilogue of one tile runs under the main loop of the next.
+//   warp 0      TMA producer (dY and X boxes of every K block of 64 tokens)
+//   warp 1      UMMA issuer, owner of the tensor-memory allocation
+//   warps 2..9  epilogue: thread = (row j, half of the tile's columns)
 template <int TN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant__ CUtensorMap tmap_x,
@@ -42,6 +48,8 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
     constexpr uint32_t kIdesc = ptx::make_idesc_bf16(kBlockM, TN, 1, 1);
     constexpr int HN = TN / 2;
     constexpr int NCH = HN / 32;
+    constexpr uint32_t kAccCols = TmemCols<TN>::value;
+    constexpr uint32_t kTmemCols = 2 * kAccCols;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -53,26 +61,36 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
     ctl.full = ctl_base;
     ctl.aready = 0;
     ctl.empty = ctl_base + 8 * STAGES;
-    ctl.accum = ctl_base + 16 * STAGES;
-    ctl.spare = ctl.accum + 8;
-    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 16 * STAGES + 16);
-    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 16 * STAGES + 20);
+    ctl.accum = ctl_base + 16 * STAGES;         // + 8c : accumulator c complete
+    const uint32_t acc_empty = ctl.accum + 16;  // + 8c : accumulator c drained
+    ctl.spare = ctl.accum + 32;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 16 * STAGES + 40);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 16 * STAGES + 44);
     ctl.device_flag = &g_timeout_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int j0 = blockIdx.x * kBlockM;
-    const int k0 = blockIdx.y * TN;
-    const int kb_begin = blockIdx.z * p.kb_per_split;
-    const int kb_end = min(p.num_kb, kb_begin + p.kb_per_split);
-    const int iters = kb_end - kb_begin;
+    const int num_tiles = p.m_tiles * p.n_tiles * p.splits;
+    // row tile fastest: CTAs running together share the X boxes of a column tile in L2
+    auto tile_coords = [&](int tile, int& j0, int& k0, int& z, int& kb_begin, int& iters) {
+        const int mt = tile % p.m_tiles;
+        const int rest = tile / p.m_tiles;
+        j0 = mt * kBlockM;
+        k0 = (rest % p.n_tiles) * TN;
+        z = rest / p.n_tiles;
+        kb_begin = z * p.kb_per_split;
+        iters = min(p.num_kb, kb_begin + p.kb_per_split) - kb_begin;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(ctl.full + 8 * s, 1);
             ptx::mbar_init(ctl.empty + 8 * s, 1);
         }
-        ptx::mbar_init(ctl.accum, 1);
+        for (int c = 0; c < 2; ++c) {
+            ptx::mbar_init(ctl.accum + 8 * c, 1);
+            ptx::mbar_init(acc_empty + 8 * c, kWorkerWarps);
+        }
         ptx::mbar_init(ctl.spare, 1);
         *ctl.abort_flag = 0;
         ptx::fence_mbar_init();
@@ -80,7 +98,7 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
         ptx::prefetch_tmap(&tmap_x);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), TmemCols<TN>::value);
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t*>(tmem_holder)), kTmemCols);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
@@ -91,126 +109,161 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
     if (warp == 0) {
         if (lane == 0) {
             bool ok = true;
-            int issued = 0;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
-                ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 11);
-                if (!ok) break;
-                const uint32_t sa = smem_base + s * kStageBytes;
-                const int tok = (kb_begin + it) * kBlockK;
-                ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kStageBytes);
-                // A: two blocks of 64 rows j (inner) x 64 tokens; B: TN/64 blocks of 64 k x 64 tokens
-                ptx::tma_load_2d(sa, &tmap_dy, j0, tok, ctl.full + 8 * s);
-                ptx::tma_load_2d(sa + 8192, &tmap_dy, j0 + 64, tok, ctl.full + 8 * s);
+            int s = 0, in_flight = 0;
+            uint32_t ph = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int j0, k0, z, kb_begin, iters;
+                tile_coords(tile, j0, k0, z, kb_begin, iters);
+                for (int it = 0; it < iters; ++it) {
+                    ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 11);
+                    if (!ok) break;
+                    const uint32_t sa = smem_base + s * kStageBytes;
+                    const int tok = (kb_begin + it) * kBlockK;
+                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kStageBytes);
+                    // A: two blocks of 64 rows j (inner) x 64 tokens; B: TN/64 blocks of 64 k x 64 tokens
+                    ptx::tma_load_2d(sa, &tmap_dy, j0, tok, ctl.full + 8 * s);
+                    ptx::tma_load_2d(sa + 8192, &tmap_dy, j0 + 64, tok, ctl.full + 8 * s);
 #pragma unroll
-                for (int b = 0; b < TN / 64; ++b)
-                    ptx::tma_load_2d(sa + kABytes + b * 8192, &tmap_x, k0 + b * 64, tok, ctl.full + 8 * s);
-                issued = it + 1;
+                    for (int b = 0; b < TN / 64; ++b)
+                        ptx::tma_load_2d(sa + kABytes + b * 8192, &tmap_x, k0 + b * 64, tok, ctl.full + 8 * s);
+                    in_flight = min(in_flight + 1, STAGES);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
             }
             if (!ok) {
-                for (int it = max(0, issued - STAGES); it < issued; ++it)
-                    wait_bar(ctl.full + 8 * (it % STAGES), (it / STAGES) & 1, ctl, 12);
+                int bs = s;
+                uint32_t bph = ph;
+                for (int i = 0; i < in_flight; ++i) {
+                    if (bs == 0) { bs = STAGES; bph ^= 1u; }
+                    --bs;
+                    wait_bar(ctl.full + 8 * bs, bph, ctl, 12);
+                }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1;
+        // the whole warp walks the loop (uniform control flow), one elected lane issues
+        bool ok = true;
+        int s = 0, lt = 0;
+        uint32_t ph = 0;
+        // descriptor halves (128-byte swizzle, MN-major: leading offset 8192 B between blocks of 64
+        // rows, stride 1024 B between groups of eight token lines); a UMMA steps the start by 2048 B
+        constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+        constexpr uint32_t kLoExtra = (8192u >> 4) << 16;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+            int j0, k0, z, kb_begin, iters;
+            tile_coords(tile, j0, k0, z, kb_begin, iters);
+            const int acc = lt & 1;
+            ok = wait_bar(acc_empty + 8 * acc, (uint32_t)((lt >> 1) & 1) ^ 1u, ctl, 17);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
+            for (int it = 0; it < iters; ++it) {
                 ok = wait_bar(ctl.full + 8 * s, ph, ctl, 13);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t sa = smem_base + s * kStageBytes;
-                const uint32_t sb = sa + kABytes;
+                if (ptx::elect_one()) {
+                    const uint32_t a_lo = (((smem_base + (uint32_t)s * kStageBytes) >> 4) & 0x3FFFu) | kLoExtra;
+                    const uint32_t b_lo = a_lo + (kABytes >> 4);
 #pragma unroll
-                for (int kk = 0; kk < kBlockK / 16; ++kk) {
-                    const uint64_t da = ptx::make_smem_desc(sa + kk * 2048, 8192, 1024);
-                    const uint64_t db = ptx::make_smem_desc(sb + kk * 2048, 8192, 1024);
-                    ptx::umma_bf16(tmem_base, da, db, kIdesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBlockK / 16; ++kk)
+                        ptx::umma_f16_halves(d_tmem, a_lo + kk * (2048u >> 4), kHi, b_lo + kk * (2048u >> 4), kHi, kIdesc,
+                                             (it > 0 || kk > 0) ? 1u : 0u);
+                    ptx::umma_commit(ctl.empty + 8 * s);
                 }
-                ptx::umma_commit(ctl.empty + 8 * s);
+                __syncwarp();
+                if (++s == STAGES) { s = 0; ph ^= 1u; }
             }
-            if (ok) {
-                ptx::umma_commit(ctl.accum);
-            } else {
-                ptx::umma_commit(ctl.spare);
-                wait_bar(ctl.spare, 0, ctl, 15);
-            }
+            if (ok && ptx::elect_one()) ptx::umma_commit(ctl.accum + 8 * acc);
+            __syncwarp();
+        }
+        if (!ok) {
+            if (ptx::elect_one()) ptx::umma_commit(ctl.spare);
+            __syncwarp();
+            wait_bar(ctl.spare, 0, ctl, 15);
         }
     } else {
         // ---------------- epilogue: thread = (row j, HN columns of the tile)
         const int quarter = warp & 3;
         const int half = (warp - kWorkerWarp0) >> 2;
-        const int j = j0 + quarter * 32 + lane;
-        const bool j_ok = j < p.d_out;
-        const int kbase = k0 + half * HN;
-        const int subtile = blockIdx.y * 2 + half;
         const long long plane_words = (long long)p.d_out * p.pitch;
+        bool ok = true;
+        int lt = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+            int j0, k0, z, kb_begin, iters;
+            tile_coords(tile, j0, k0, z, kb_begin, iters);
+            const int acc = lt & 1;
+            const int j = j0 + quarter * 32 + lane;
+            const bool j_ok = j < p.d_out;
+            const int kbase = k0 + half * HN;
+            const int subtile = (k0 / TN) * 2 + half;
 
-        // the sign words do not depend on the accumulator: fetch them while the main loop runs
-        uint32_t nw[NCH][BCQ_MAX_Q];
-#pragma unroll
-        for (int ch = 0; ch < NCH; ++ch) {
-            const int kw = (kbase >> 5) + ch;
-#pragma unroll
-            for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                const bool act = (i < p.q) && ((p.plane_mask >> i) & 1u) && j_ok && (kw < p.pitch);
-                nw[ch][i] = act ? ~__ldg(p.bits + i * plane_words + (long long)j * p.pitch + kw) : 0u;
-            }
-        }
-
-        bool ok = wait_bar(ctl.accum, 0, ctl, 16);
-        if (ok && kbase < p.d_in) {
-            ptx::tc_fence_after_sync();
-            const int c_first = min(kbase / p.g, p.G - 1);
-            float acc[BCQ_MAX_Q];
-#pragma unroll
-            for (int i = 0; i < BCQ_MAX_Q; ++i) acc[i] = 0.0f;
-            int cur_c = c_first;
-            auto flush = [&](int c) {
-                if (!j_ok) return;
-                const int slot = c - c_first;
-#pragma unroll
-                for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                    if (i < p.q && ((p.plane_mask >> i) & 1u)) {
-                        const long long idx =
-                            ((((long long)blockIdx.z * p.n_subtiles + subtile) * p.q + i) * p.slots + slot) *
-                                p.d_out + j;
-                        p.partial[idx] = acc[i];
-                    }
-                }
-            };
+            // the sign words do not depend on the accumulator: fetch them while the main loop runs
+            uint32_t nw[NCH][BCQ_MAX_Q];
 #pragma unroll
             for (int ch = 0; ch < NCH; ++ch) {
-                const int kg = kbase + ch * 32;
-                if (kg < p.d_in) {  // uniform in the warp
-                    const int c = min(kg / p.g, p.G - 1);
-                    if (c != cur_c) {
-                        flush(cur_c);
-                        cur_c = c;
+                const int kw = (kbase >> 5) + ch;
 #pragma unroll
-                        for (int i = 0; i < BCQ_MAX_Q; ++i) acc[i] = 0.0f;
-                    }
-                    uint32_t v[32];
-                    ptx::tmem_ld_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) +
-                                         (uint32_t)(half * HN + ch * 32), v);
-                    ptx::tmem_ld_wait();
+                for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                    const bool act = (i < p.q) && ((p.plane_mask >> i) & 1u) && j_ok && (kw < p.pitch);
+                    nw[ch][i] = act ? ~__ldg(p.bits + i * plane_words + (long long)j * p.pitch + kw) : 0u;
+                }
+            }
+
+            ok = wait_bar(ctl.accum + 8 * acc, (uint32_t)(lt >> 1) & 1u, ctl, 16, 512u);
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            if (kbase < p.d_in) {
+                const int c_first = min(kbase / p.g, p.G - 1);
+                float accs[BCQ_MAX_Q];
+#pragma unroll
+                for (int i = 0; i < BCQ_MAX_Q; ++i) accs[i] = 0.0f;
+                int cur_c = c_first;
+                auto flush = [&](int c) {
+                    if (!j_ok) return;
+                    const int slot = c - c_first;
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) {
                         if (i < p.q && ((p.plane_mask >> i) & 1u)) {
-                            const uint32_t w = nw[ch][i];
-                            float s = 0.0f;
+                            const long long idx =
+                                ((((long long)z * p.n_subtiles + subtile) * p.q + i) * p.slots + slot) * p.d_out + j;
+                            p.partial[idx] = accs[i];
+                        }
+                    }
+                };
 #pragma unroll
-                            for (int b = 0; b < 32; ++b)
-                                s += __uint_as_float(v[b] ^ ((w << (31 - b)) & 0x80000000u));
-                            acc[i] += s;
+                for (int ch = 0; ch < NCH; ++ch) {
+                    const int kg = kbase + ch * 32;
+                    if (kg < p.d_in) {  // uniform in the warp
+                        const int c = min(kg / p.g, p.G - 1);
+                        if (c != cur_c) {
+                            flush(cur_c);
+                            cur_c = c;
+#pragma unroll
+                            for (int i = 0; i < BCQ_MAX_Q; ++i) accs[i] = 0.0f;
+                        }
+                        uint32_t v[32];
+                        ptx::tmem_ld_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * kAccCols +
+                                             (uint32_t)(half * HN + ch * 32), v);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                            if (i < p.q && ((p.plane_mask >> i) & 1u)) {
+                                const uint32_t w = nw[ch][i];
+                                float sum = 0.0f;
+#pragma unroll
+                                for (int b = 0; b < 32; ++b)
+                                    sum += __uint_as_float(v[b] ^ ((w << (31 - b)) & 0x80000000u));
+                                accs[i] += sum;
+                            }
                         }
                     }
                 }
+                flush(cur_c);
             }
-            flush(cur_c);
+            // the accumulator may be overwritten by the tile after next
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(acc_empty + 8 * acc);
         }
     }
 
@@ -218,7 +271,7 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, TmemCols<TN>::value);
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -352,23 +405,25 @@ extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, in
     p.G = (int)bcq_num_groups(d_in, g);
     p.pitch = (int)bcq_pitch_words(d_in);
     p.n = n; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
+    p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
     p.n_subtiles = pl.n_subtiles; p.slots = pl.slots; p.plane_mask = plane_mask;
     p.bits = bits; p.partial = reinterpret_cast<float*>(ws);
     cudaStream_t s = (cudaStream_t)stream;
-    dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.n_tiles, (unsigned)pl.splits);
+    // persistent, one CTA per SM; every CTA gets the same number of tiles (as many as the busiest
+    // would get anyway), which leaves whole SMs to other kernels instead of a ragged last wave
+    const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
+    const int per_cta = ceil_div(tiles, sm_count());
+    const unsigned grid = (unsigned)ceil_div(tiles, per_cta);
     if (pl.TN == 256) {
         auto kern = dalpha_kernel<256, stages_for<256>()>;
-        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem_for<256>()));
+        if ((st = ensure_dynamic_smem(kern, smem_for<256>())) != BCQ_OK) return st;
         kern<<<grid, kThreads, smem_for<256>(), s>>>(tm_dy, tm_x, p);
-    bcq::count_launch();
     } else {
         auto kern = dalpha_kernel<128, stages_for<128>()>;
-        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem_for<128>()));
+        if ((st = ensure_dynamic_smem(kern, smem_for<128>())) != BCQ_OK) return st;
         kern<<<grid, kThreads, smem_for<128>(), s>>>(tm_dy, tm_x, p);
-    bcq::count_launch();
     }
+    bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
     const long long rblocks = (long long)q * p.G * ((d_out + 31) / 32);
     dalpha_reduce_kernel<<<(unsigned)rblocks, 256, 0, s>>>(

@@ -696,22 +696,11 @@ DecPackedPlan plan_decode_packed(const PackLayout& L, int n) {
     return pl;
 }
 
-template <typename Kern>
-bcq_status ensure_smem(Kern kern, size_t bytes) {
-    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
-    return BCQ_OK;
-}
-
 template <int Q>
 bcq_status launch_decode_packed(const DecPackedParams& p, const DecPackedPlan& pl, cudaStream_t s) {
     auto kern = decode_packed_kernel<Q>;
-    static int configured[64] = {};
-    int dev = 0;
-    BCQ_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || configured[dev] < (int)pl.smem) {
-        BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
-        if (dev >= 0 && dev < 64) configured[dev] = (int)pl.smem;
-    }
+    bcq_status st0 = ensure_dynamic_smem(kern, pl.smem);
+    if (st0 != BCQ_OK) return st0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)pl.ctas);
     cfg.blockDim = dim3(kDpThreads);

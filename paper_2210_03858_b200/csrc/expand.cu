@@ -1496,7 +1496,8 @@ template <int MODE, int TN, int QM>
 bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
                          cudaStream_t stream) {
     auto kern = expand_gemm_kernel<MODE, TN, QM>;
-    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem));
+    bcq_status st0 = ensure_dynamic_smem(kern, pl.smem);
+    if (st0 != BCQ_OK) return st0;
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
     // persistent, at most one CTA per SM; with more tiles than SMs every CTA gets the same number of
     // tiles (as many as the busiest would get anyway): fewer CTAs pay the prologue, more epilogues
@@ -1640,7 +1641,8 @@ bcq_status launch_decode(const CUtensorMap& tm_bits, const DecodeParams& p, cons
                          cudaStream_t s) {
     constexpr size_t smem = (size_t)kDecStages * StageLayout<MODE_FWD, kDecTN, QM>::kStageBytes + 1024 + 512;
     auto kern = decode_kernel<QM>;
-    BCQ_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    bcq_status st0 = ensure_dynamic_smem(kern, smem);
+    if (st0 != BCQ_OK) return st0;
     dim3 grid((unsigned)pl.m_tiles, (unsigned)pl.splits);
     kern<<<grid, kThreads, smem, s>>>(tm_bits, p);
     bcq::count_launch();

@@ -78,6 +78,14 @@ struct TmemCols {
 // host helpers
 // ------------------------------------------------------------------------------------------
 
+// Raises a kernel's dynamic shared memory limit, once per (kernel, device) (the attribute call is
+// not free, and callers that launch eagerly would pay it on every call).  Defined in api.cu.
+bcq_status ensure_dynamic_smem_impl(const void* kern, size_t bytes);
+template <typename Kern>
+inline bcq_status ensure_dynamic_smem(Kern kern, size_t bytes) {
+    return ensure_dynamic_smem_impl(reinterpret_cast<const void*>(kern), bytes);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
