@@ -485,13 +485,13 @@ struct ExpandParams {
     int kb_per_split;
     int splits;
     int m_tiles, n_tiles;
-    // pipeline geometry (chosen on the host from q and g)
-    int stages;            // operand slots: a multiple of the number of worker groups, <= 8
-    int aux_slots;         // ring of plane-word / scale chunks: same rule, >= stages; filled ahead of the operand slots
+    int tn;                // token tile width
+    uint32_t acc_cols;     // tensor-memory columns per accumulator
+    // pipeline geometry (chosen on the host)
+    int a_slots;           // ring of expanded weight tiles (16 KiB each), >= the number of worker groups
+    int b_slots;           // ring of activation tiles (TN x 128 B each), filled by TMA
     int epi_bufs;          // staging buffers per epilogue warp: 1 or 2
-    uint32_t bits_bytes;   // q KiB: the stage's plane words
-    uint32_t alpha_bytes;  // q * rows * 4: the scales of one group for the stage's rows
-    int alpha_parts;       // groups a stage (fwd: 64 k) or a tile (dX: 128 k) can touch: 1, 2 or 4
+    uint32_t chunk_words;  // words of one stage's chunk of the regrouped planes
     const uint32_t* bits_t;      // regrouped plane words (see PrepParams)
     const float* alpha_t;        // regrouped scales
     const float* bias;           // fwd only, may be null
@@ -522,72 +522,72 @@ struct StageLayout {
 // Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
 // running at the same time share activation tiles in L2).  32 warps:
 //   warps 0..23   workers in three groups of eight; group g takes the pipeline stages whose running
-//                 index is g mod 3.  A thread expands 32 weights of one row per stage (one plane
-//                 word per plane), so a group rebuilds one 128 x 64 weight tile.  The expansion is
-//                 a chain of dependent shifts, masks and PRMTs, so it is the number of warps in
-//                 flight, not the issue rate, that bounds it
+//                 index is g mod 3.  A thread expands 32 weights of one row per stage, so a group
+//                 rebuilds one 128 x 64 weight tile.  The thread reads its selector codes (or plane
+//                 words) and scales straight from the regrouped arrays in global memory, one task
+//                 ahead of the one it expands, so the loads are hidden behind a whole turn of the
+//                 group
 //   warp 24       UMMA issuer, owner of the tensor-memory allocation (two accumulators)
-//   warps 25..27  producers: the activation tile of a stage (TMA), its plane words and its scales
-//                 (bulk copies of the chunks the pre-pass regrouped)
+//   warp 25       producer of the activation tiles (TMA)
 //   warps 28..31  epilogue: drain one accumulator while the main loop fills the other (warp w
 //                 reaches the tensor-memory lanes 32 * (w % 4) .. + 31)
-// Shared memory: STAGES x | A tile 16 KiB | B tile TN x 128 B |, the epilogue's staging, AUXS x
-// | plane words | scales | group indices |, then barriers and output scales.
+// Shared memory: a ring of weight tiles (16 KiB each; few, the workers refill one as soon as the
+// tensor core is done with it), a deeper ring of activation tiles (TN x 128 B each; a TMA load
+// takes about a microsecond to land), the epilogue's staging, barriers and output scales.
 constexpr int kPfGroups = 3;
 constexpr int kPfGroupWarps = 8;
 constexpr int kPfWorkerWarps = kPfGroups * kPfGroupWarps;  // 24
 constexpr int kPfMmaWarp = kPfWorkerWarps;                 // 24
-constexpr int kPfProdWarp0 = kPfMmaWarp + 1;               // 25, 26, 27
-constexpr int kPfEpiWarp0 = kPfProdWarp0 + 3;              // 28
+constexpr int kPfProdWarp = kPfMmaWarp + 1;                // 25
+constexpr int kPfEpiWarp0 = 28;
 constexpr int kPfEpiWarps = 4;
 constexpr int kPfWarps = kPfEpiWarp0 + kPfEpiWarps;        // 32
 constexpr int kPfThreads = kPfWarps * 32;                  // 1024
 static_assert(kPfEpiWarp0 % 4 == 0, "epilogue warp e must sit on tensor-memory lane quarter e");
 __device__ __forceinline__ int pf_worker_index(int warp) { return warp < kPfWorkerWarps ? warp : -1; }
 __device__ __forceinline__ int pf_epilogue_index(int warp) { return warp >= kPfEpiWarp0 ? warp - kPfEpiWarp0 : -1; }
-constexpr int kPfMaxStages = 8;
+constexpr int kPfMaxSlots = 8;                                // per ring
+constexpr uint32_t kPfGroupBar0 = 4;                           // named barriers 4, 5, 6: one per worker group
 constexpr uint32_t kPfCtlBytes = 384;                          // barriers, TMEM handle, abort flag
 constexpr uint32_t kPfScaleBytes = 256 * 4;                    // [TN] output scales of the tile being drained
 constexpr uint32_t kPfStagingBuf = kPfEpiWarps * 1024;         // per epilogue warp one 1 KiB buffer of 32 rows x 16 bf16 (8 fp32) tokens; one or two such sets
 
-template <int MODE, int TN, int QM>
+template <int MODE, int QM>
 __global__ void __launch_bounds__(kPfThreads, 1)
 expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_constant__ CUtensorMap tmap_out,
                    const ExpandParams p) {
-    constexpr uint32_t kBBytes = TN * kBlockK * 2;
-    constexpr uint32_t kStageBytes = kABytes + kBBytes;
-    constexpr uint32_t kTmemCols = 2 * TmemCols<TN>::value;
+    const int TN = p.tn;                                   // token tile: a multiple of 16, <= 256
+    const uint32_t kBBytes = (uint32_t)TN * kBlockK * 2;
+    const uint32_t kAccCols = p.acc_cols;                  // tensor-memory columns of one accumulator
+    const uint32_t kTmemCols = 2 * kAccCols;               // a power of two >= 32
     constexpr int kRows = (MODE == MODE_FWD) ? 128 : 64;  // weight rows of one stage
-    constexpr int kUnit = (MODE == MODE_FWD) ? 2 : 4;     // plane words per row and stage
+    constexpr int kUnit = (MODE == MODE_FWD) ? 2 : 4;     // 32-weight blocks per row and stage
     constexpr int NW = NumWords<QM>::value;
     // fp16 x fp16 -> fp32; A is MN-major for dX
-    constexpr uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
-                                ~((1u << 7) | (1u << 10));
+    const uint32_t kIdesc = (ptx::make_idesc_bf16(kBlockM, TN, MODE == MODE_BWDX ? 1 : 0, 0)) &
+                            ~((1u << 7) | (1u << 10));
 
     extern __shared__ uint8_t smem_raw[];
-    const int STAGES = p.stages;
+    const int NA = p.a_slots, NB = p.b_slots;
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t staging_base = smem_base + STAGES * kStageBytes;  // 1 KiB aligned: the output boxes are swizzled
-    const int AUXS = p.aux_slots;
+    const uint32_t b_base = smem_base + NA * kABytes;
+    const uint32_t staging_base = b_base + NB * kBBytes;  // 1 KiB aligned: the output boxes are swizzled
     const uint32_t staging_bytes = (uint32_t)p.epi_bufs * kPfStagingBuf;
-    const uint32_t aux_base = staging_base + staging_bytes;
-    const uint32_t kAuxBytes = p.bits_bytes + p.alpha_parts * p.alpha_bytes;
-    const uint32_t ctl_base = aux_base + AUXS * kAuxBytes;
-    uint8_t* ctl_gen = smem_gen + STAGES * kStageBytes + staging_bytes + AUXS * kAuxBytes;
+    const uint32_t ctl_base = staging_base + staging_bytes;
+    uint8_t* ctl_gen = smem_gen + NA * kABytes + NB * kBBytes + staging_bytes;
 
     Ctl ctl;
-    ctl.full = ctl_base;
-    ctl.aready = ctl_base + 8 * kPfMaxStages;
-    ctl.empty = ctl_base + 16 * kPfMaxStages;
-    ctl.accum = ctl_base + 24 * kPfMaxStages;   // accumulator full [2]
+    ctl.aready = ctl_base;                      // + 8*s : the workers have written weight slot s
+    ctl.empty = ctl_base + 8 * kPfMaxSlots;     // + 8*s : the UMMAs that read weight slot s are done
+    ctl.full = ctl_base + 16 * kPfMaxSlots;     // + 8*s : the activation tile of slot s has landed
+    const uint32_t b_empty = ctl_base + 24 * kPfMaxSlots;  // + 8*s : the UMMAs that read activation slot s are done
+    ctl.accum = ctl_base + 32 * kPfMaxSlots;    // accumulator full [2]
     const uint32_t acc_empty = ctl.accum + 16;  // accumulator drained [2]
     ctl.spare = acc_empty + 16;
-    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 24 * kPfMaxStages + 40);
-    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 24 * kPfMaxStages + 44);
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(ctl_gen + 32 * kPfMaxSlots + 40);
+    ctl.abort_flag = reinterpret_cast<volatile int*>(ctl_gen + 32 * kPfMaxSlots + 44);
     ctl.device_flag = &g_timeout_flag;
-    const uint32_t wfull = ctl_base + 256;   // + 8*a : plane words and scales of aux slot a have landed
-    const uint32_t wempty = ctl_base + 320;  // + 8*a : the worker group that used aux slot a has read it
     float* scale = reinterpret_cast<float*>(ctl_gen + kPfCtlBytes);  // [TN]: 1 / (weight scale * token scale)
     const uint32_t scale_addr = ctl_base + kPfCtlBytes;
 
@@ -597,12 +597,12 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     if (warp == 0) {
         // the barriers are initialised by the lanes of one warp side by side (one after the other
         // they cost a few tenths of a microsecond before any copy can start)
-        if (lane < STAGES) {
-            ptx::mbar_init(ctl.aready + 8 * lane, kPfGroupWarps + 1);  // both operands: the worker warps and the activation tile
+        if (lane < NA) {
+            ptx::mbar_init(ctl.aready + 8 * lane, kPfGroupWarps);
             ptx::mbar_init(ctl.empty + 8 * lane, 1);
-        } else if (lane >= 8 && lane < 8 + AUXS) {
-            ptx::mbar_init(wfull + 8 * (lane - 8), 1 + p.alpha_parts);  // plane words; each part of the scales
-            ptx::mbar_init(wempty + 8 * (lane - 8), kPfGroupWarps);
+        } else if (lane >= 8 && lane < 8 + NB) {
+            ptx::mbar_init(ctl.full + 8 * (lane - 8), 1);
+            ptx::mbar_init(b_empty + 8 * (lane - 8), 1);
         } else if (lane >= 16 && lane < 18) {
             ptx::mbar_init(ctl.accum + 8 * (lane - 16), 1);
             ptx::mbar_init(acc_empty + 8 * (lane - 16), kPfEpiWarps);
@@ -674,73 +674,24 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
     constexpr int kPfHelpers = 1 + kPfWorkerWarps / 4;  // 7
     auto is_last_tile = [&](int tile) { return tile + (int)gridDim.x >= num_tiles; };
 
-    if (warp >= kPfProdWarp0 && warp < kPfEpiWarp0) {
-        // ---------------- producers.  Issuing one copy costs a thread a few hundred cycles, so
-        // the three kinds of copies of a stage come from three warps, each walking the stages on
-        // its own: the activation tile (TMA), the plane words, the scales with the group indices
-        // (lane a = part a).  Each arrives on the barrier of what it fills with the bytes it brings.
-        const int role = warp - kPfProdWarp0;
-        const int parts = (role == 2) ? p.alpha_parts : 1;
-        if (lane < parts) {
+    if (warp == kPfProdWarp) {
+        // ---------------- producer: the activation tile of every stage (TMA), into a ring of its
+        // own that runs as far ahead of the tensor core as shared memory allows
+        if (lane == 0) {
             bool ok = true;
-            // role 0 cycles over the operand slots (freed by the UMMAs that read them), roles 1 and 2
-            // over the longer ring of weight chunks (freed by the workers as soon as they have read one)
-            const int ring = (role == 0) ? STAGES : AUXS;
-            const uint32_t free_bar = (role == 0) ? ctl.empty : wempty;
-            const uint32_t fill_bar = (role == 0) ? ctl.aready : wfull;
             int s = 0, in_flight = 0;
             uint32_t ph = 0;
-            const int span = ((MODE == MODE_FWD) ? 64 : 128) / p.alpha_parts;  // k covered by one part
-            const uint32_t bits_words = p.bits_bytes >> 2, alpha_words = p.alpha_bytes >> 2;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int m0, t0, z, kb_begin, iters;
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
-                const int mt = m0 >> 7;
-                // plane words: chunk [m_tile][kb] (fwd) or [u][jb] (dX), consecutive in kb
-                const uint32_t* bits_src = p.bits_t + ((long long)mt * p.num_kb + kb_begin) * bits_words;
-                // group index of this lane's part: for dX fixed by the tile; for the forward it
-                // advances with k (kept incrementally, no division in the stage loop)
-                int kpos = ((MODE == MODE_FWD) ? kb_begin * kBlockK : m0) + lane * span;
-                int c = min(kpos / p.g, p.G - 1);
-                int next_edge = (c + 1) * p.g;  // first k of the next group
-                int hist0 = -1, hist1 = -1, hist2 = -1;  // group index of this part 3, 2, 1 stages ago
-                static_assert(kPfGroups == 3, "the history covers three stages");
-                // scales: block [m_tile][G] (fwd) or [jb][G] (dX) of alpha_words each
-                const float* alpha_src = p.alpha_t + (long long)((MODE == MODE_FWD) ? mt : kb_begin) * p.G * alpha_words;
                 for (int it = 0; it < iters; ++it) {
-                    ok = wait_bar(free_bar + 8 * s, ph ^ 1u, ctl, 1);
+                    ok = wait_bar(b_empty + 8 * s, ph ^ 1u, ctl, 1);
                     if (!ok) break;
-                    const uint32_t bar = fill_bar + 8 * s;
-                    if (role == 0) {
-                        ptx::mbar_arrive_expect_tx(bar, kBBytes);
-                        ptx::tma_load_2d(smem_base + s * kStageBytes + kABytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
-                    } else if (role == 1) {
-                        ptx::mbar_arrive_expect_tx(bar, p.bits_bytes);
-                        ptx::bulk_load(aux_base + s * kAuxBytes, bits_src, p.bits_bytes, bar);
-                        bits_src += bits_words;
-                    } else {
-                        // a worker rebuilds its lookup table when the group index differs from the
-                        // one of its previous stage (kPfGroups stages back) and at its first stage
-                        // of a tile; for dX every stage brings other rows.  Only then does it read
-                        // the scales, so only then are they copied.
-                        const bool need = (MODE == MODE_BWDX) || (QM == QM_GENERIC) || (c != hist0);  // q > 4: no table, read every stage
-                        hist0 = hist1; hist1 = hist2; hist2 = c;
-                        if (need) {
-                            ptx::mbar_arrive_expect_tx(bar, p.alpha_bytes);
-                            ptx::bulk_load(aux_base + s * kAuxBytes + p.bits_bytes + lane * p.alpha_bytes,
-                                           alpha_src + (long long)c * alpha_words, p.alpha_bytes, bar);
-                        } else {
-                            ptx::mbar_arrive(bar);
-                        }
-                        if (MODE == MODE_FWD) {
-                            kpos += kBlockK;
-                            while (kpos >= next_edge && c < p.G - 1) { ++c; next_edge += p.g; }
-                        } else {
-                            alpha_src += (long long)p.G * alpha_words;  // next block of 64 rows
-                        }
-                    }
-                    in_flight = min(in_flight + 1, ring);
-                    if (++s == ring) { s = 0; ph ^= 1u; }
+                    const uint32_t bar = ctl.full + 8 * s;
+                    ptx::mbar_arrive_expect_tx(bar, kBBytes);
+                    ptx::tma_load_2d(b_base + s * kBBytes, &tmap_b, (kb_begin + it) * kBlockK, t0, bar);
+                    in_flight = min(in_flight + 1, NB);
+                    if (++s == NB) { s = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
@@ -749,9 +700,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 int bs = s;
                 uint32_t bph = ph;
                 for (int i = 0; i < in_flight; ++i) {
-                    if (bs == 0) { bs = ring; bph ^= 1u; }
+                    if (bs == 0) { bs = NB; bph ^= 1u; }
                     --bs;
-                    wait_bar(fill_bar + 8 * bs, bph, ctl, 2);
+                    wait_bar(ctl.full + 8 * bs, bph, ctl, 2);
                 }
             }
         }
@@ -759,8 +710,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // ---------------- UMMA issuer: the whole warp walks the stages and waits on the barriers
         // (warp-uniform control flow); one elected lane issues
         bool ok = true;
-        int s = 0, lt = 0;
-        uint32_t ph = 0;
+        int sa = 0, sb = 0, lt = 0;
+        uint32_t pha = 0, phb = 0;
         // shared-memory descriptor halves (128-byte swizzle, version 1): low = start address >> 4 and
         // leading offset >> 4 at bit 16, high = stride offset >> 4, version at bit 14, swizzle at bit 29
         constexpr uint32_t kHiCommon = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -769,6 +720,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         constexpr uint32_t kBLoExtra = (16u >> 4) << 16;
         constexpr uint32_t kAStep = (MODE == MODE_FWD) ? (32u >> 4) : (2048u >> 4);
         const uint32_t a_lo0 = ((smem_base >> 4) & 0x3FFFu) | kALoExtra;
+        const uint32_t b_lo0 = ((b_base >> 4) & 0x3FFFu) | kBLoExtra;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
             int m0, t0, z, kb_begin, iters;
             tile_coords(tile, m0, t0, z, kb_begin, iters);
@@ -777,24 +729,26 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)acc * TmemCols<TN>::value;
+            const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
             for (int it = 0; it < iters; ++it) {
-                ok = wait_bar(ctl.aready + 8 * s, ph, ctl, 4);  // both operands of the stage are in place
+                ok = wait_bar(ctl.full + 8 * sb, phb, ctl, 4, 32u) && wait_bar(ctl.aready + 8 * sa, pha, ctl, 3, 32u);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 if (ptx::elect_one()) {
                     // descriptors: only the start-address field changes, by 32 bytes (K-major) or
                     // 2048 bytes (MN-major A) per UMMA
-                    const uint32_t a_lo = a_lo0 + (uint32_t)s * (kStageBytes >> 4);
-                    const uint32_t b_lo = a_lo + (kABytes >> 4) - kALoExtra + kBLoExtra;
+                    const uint32_t a_lo = a_lo0 + (uint32_t)sa * (kABytes >> 4);
+                    const uint32_t b_lo = b_lo0 + (uint32_t)sb * (kBBytes >> 4);
 #pragma unroll
                     for (int kk = 0; kk < kBlockK / 16; ++kk)
                         ptx::umma_f16_halves(d_tmem, a_lo + kk * kAStep, kAHi, b_lo + kk * 2, kBHi, kIdesc,
                                              (it > 0 || kk > 0) ? 1u : 0u);
-                    ptx::umma_commit(ctl.empty + 8 * s);
+                    ptx::umma_commit(ctl.empty + 8 * sa);
+                    ptx::umma_commit(b_empty + 8 * sb);
                 }
                 __syncwarp();
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (++sa == NA) { sa = 0; pha ^= 1u; }
+                if (++sb == NB) { sb = 0; phb ^= 1u; }
             }
             if (ok && ptx::elect_one()) ptx::umma_commit(ctl.accum + 8 * acc);
             __syncwarp();
@@ -820,101 +774,161 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const uint32_t line_off = (MODE == MODE_FWD) ? row * 128 : ((part >> 1) * 8192) + row * 128;
         const uint32_t lx = row & 7;
         const uint32_t chunk0 = (MODE == MODE_FWD) ? part * 4 : (part & 1) * 4;
-        // which of the stage's alpha parts covers this thread's 32 k
-        const int apart = (MODE == MODE_FWD) ? (p.alpha_parts == 2 ? part : 0)
-                                             : (p.alpha_parts == 4 ? part : (p.alpha_parts == 2 ? (part >> 1) : 0));
-        const uint32_t w_off = (uint32_t)(row * kUnit + part) * 4;                        // + i * kRows * kUnit * 4 (q > 4: plane words)
         constexpr int NWC = CodeWords<QM>::value;
-        const uint32_t c_off = (uint32_t)((row * kUnit + part) * NWC) * 4;               // q <= 4: selector codes
-        const uint32_t a_off = p.bits_bytes + apart * p.alpha_bytes + (uint32_t)row * 4;  // + i * kRows * 4
+        constexpr int NL = (QM == QM_GENERIC) ? NW : NWC;   // words a task loads
+        constexpr int NS = (QM == QM_GENERIC) ? NW : 4;     // scales a task loads
+        // the task's words within a chunk [m_tile][kb] (fwd) or [u][jb] (dX) of the regrouped planes:
+        // q <= 4 selector codes [row][block][NWC], q > 4 plane words [plane][row][block]
+        const uint32_t word_off = (QM == QM_GENERIC) ? (uint32_t)(row * kUnit + part) : (uint32_t)((row * kUnit + part) * NWC);
+        const uint32_t chunk_words = p.chunk_words;
+        const uint32_t alpha_block = (uint32_t)p.q * kRows;  // floats per (row block, group): [plane][row]
+
+        // The task stream of this thread: the stages whose running index over all tiles of the CTA
+        // is `group` mod kPfGroups.  A cursor names one of them.
+        struct Cur {
+            int tile, it, iters, kb_begin, mt;
+            int c, kpos, next_edge;  // group index of the task's 32 k (forward: advances with the stage)
+            bool fresh;              // the scales differ from the previous task's: load them, rebuild the table
+            bool valid;
+        };
+        auto enter_tile = [&](Cur& x) {
+            int m0, t0, z;
+            tile_coords(x.tile, m0, t0, z, x.kb_begin, x.iters);
+            x.mt = m0 >> 7;
+        };
+        auto locate = [&](Cur& x) {  // group index at (tile, it), from scratch
+            x.kpos = (MODE == MODE_FWD) ? (x.kb_begin + x.it) * kBlockK + part * 32 : x.mt * kBlockM + part * 32;
+            x.c = min(x.kpos / p.g, p.G - 1);
+            x.next_edge = (x.c + 1) * p.g;
+        };
+        // to the next task: kPfGroups stages on
+        auto advance = [&](Cur& x) {
+            x.it += kPfGroups;
+            bool moved = false;
+            while (x.it >= x.iters) {
+                x.it -= x.iters;
+                x.tile += gridDim.x;
+                if (x.tile >= num_tiles) { x.valid = false; return; }
+                enter_tile(x);
+                moved = true;
+            }
+            if (moved) {
+                locate(x);
+                x.fresh = true;
+            } else if (MODE == MODE_FWD) {
+                const int c0 = x.c;
+                x.kpos += kPfGroups * kBlockK;
+                while (x.kpos >= x.next_edge && x.c < p.G - 1) { ++x.c; x.next_edge += p.g; }
+                x.fresh = (QM == QM_GENERIC) || (x.c != c0);
+            } else {
+                x.fresh = true;  // dX: every stage brings other rows
+            }
+        };
+        // global loads of a task: its plane words or codes and, when they change, its scales
+        auto issue = [&](const Cur& x, uint32_t (&cv)[NL], float (&av)[NS]) {
+            const uint32_t* src = p.bits_t + ((long long)x.mt * p.num_kb + x.kb_begin + x.it) * chunk_words + word_off;
+            if (QM == QM_GENERIC) {
+#pragma unroll
+                for (int i = 0; i < NL; ++i) cv[i] = (i < p.q) ? ptx::ldg_nc_u32(src + i * (kRows * kUnit)) : 0u;
+            } else if (NWC == 4) {
+                const uint4 v = ptx::ldg_nc_v4(src);
+                cv[0] = v.x; cv[1] = v.y; cv[2] = v.z; cv[NL - 1] = v.w;
+            } else {
+#pragma unroll
+                for (int i = 0; i < NL; ++i) cv[i] = ptx::ldg_nc_u32(src + i);
+            }
+            if (x.fresh) {
+                const int blk = (MODE == MODE_FWD) ? x.mt : x.kb_begin + x.it;
+                const float* ap = p.alpha_t + ((long long)blk * p.G + x.c) * alpha_block + row;
+#pragma unroll
+                for (int i = 0; i < NS; ++i)
+                    av[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
+            }
+        };
 
         Lut lut = {0u, 0u, 0u, 0u};
         bool ok = true;
-        int s = 0, as = 0, gi = 0;  // operand slot, aux slot, running stage index mod kPfGroups
-        uint32_t ph = 0, aph = 0;
-        auto advance = [&](int k) {
-            s += k;
-            if (s >= STAGES) { s -= STAGES; ph ^= 1u; }
-            as += k;
-            if (as >= AUXS) { as -= AUXS; aph ^= 1u; }
+        int s = group;  // weight slot of the current task (NA >= kPfGroups)
+        uint32_t ph = 0;
+        // One task: wait until the UMMAs that read the slot's previous contents are done (the first
+        // warp of the group polls the barrier, the others park on a hardware barrier: a polling
+        // warp takes issue slots from the warps that expand), expand, publish.
+        auto process = [&](const Cur& x, const uint32_t (&cv)[NL], const float (&av)[NS]) -> bool {
+            if (wl == 0) wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9, 32u);  // a timeout shows in the abort flag
+            ptx::named_bar_sync(kPfGroupBar0 + group, kPfGroupWarps * 32);
+            if (*ctl.abort_flag) return false;
+            const uint32_t line = smem_base + (uint32_t)s * kABytes + line_off;
+            if (QM == QM_GENERIC) {
+                float a8[BCQ_MAX_Q];
+                uint32_t w8[BCQ_MAX_Q];
+#pragma unroll
+                for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                    a8[i] = av[i % NS] * wscale;
+                    w8[i] = cv[i % NL];
+                }
+                expand16_sum(w8, a8, p.q, line, lx, chunk0);
+#pragma unroll
+                for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
+                expand16_sum(w8, a8, p.q, line, lx, chunk0 + 2);
+            } else {
+                if (x.fresh)
+                    lut = (QM == QM_LUT4) ? build_lut(av[0] * wscale, av[1] * wscale, av[2] * wscale, av[3 % NS] * wscale)
+                                          : build_lut(av[0] * wscale, av[1] * wscale, av[2] * wscale, 0.0f);
+                uint32_t cw[NWC], S[4];
+#pragma unroll
+                for (int i = 0; i < NWC; ++i) cw[i] = cv[i % NL];
+                selectors<NWC>(cw, S);
+                expand32_codes<NWC>(S, lut, line, lx, chunk0);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
+            s += kPfGroups;
+            if (s >= NA) { s -= NA; ph ^= 1u; }
+            return true;
         };
 
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-            int m0, t0, z, kb_begin, iters;
-            tile_coords(tile, m0, t0, z, kb_begin, iters);
-            int lut_key = -1;  // group the table holds; rows change with the tile (and, for dX, the stage)
-            // group index of this thread's 32 k at its stages (forward), kept incrementally
-            int kpos = (kb_begin + ((group - gi + kPfGroups) % kPfGroups)) * kBlockK + apart * 32;
-            int cw = min(kpos / p.g, p.G - 1);
-            int next_edge = (cw + 1) * p.g;
-            // our stages of this tile are it = first, first + kPfGroups, ...
-            const int first = (group - gi + kPfGroups) % kPfGroups;
-            advance(min(first, iters));
-            for (int it = first; it < iters && ok; it += kPfGroups) {
-                ok = wait_bar(wfull + 8 * as, aph, ctl, 6);  // the chunk has landed
-                if (!ok) break;
-                const uint32_t stage = smem_base + s * kStageBytes;
-                const uint32_t aux = aux_base + as * kAuxBytes;
-                uint32_t w[NW];
-                uint32_t cv[NWC];
-                if (QM == QM_GENERIC) {
-#pragma unroll
-                    for (int i = 0; i < NW; ++i)
-                        w[i] = (i < p.q) ? ptx::ld_shared_u32(aux + w_off + i * (kRows * kUnit * 4)) : 0u;
-                } else {
-                    load_codes<NWC>(aux + c_off, cv);
-                }
-                // The aux slot is handed back only after the expansion below has consumed what was
-                // loaded from it: a load that has merely been issued may still be reading shared
-                // memory when the producer's next bulk copy (another proxy) overwrites the slot.
-                auto release_aux = [&]() {
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(wempty + 8 * as);
-                };
-                // until the UMMAs that read the operand slot's previous contents are done
-                auto acquire_slot = [&]() { return wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9); };
-                if (QM == QM_GENERIC) {
-                    float a8[BCQ_MAX_Q];
-                    uint32_t w8[BCQ_MAX_Q];
-#pragma unroll
-                    for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                        a8[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
-                        w8[i] = w[i % NW];
-                    }
-                    ok = acquire_slot();
-                    if (!ok) break;
-                    expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0);
-#pragma unroll
-                    for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
-                    expand16_sum(w8, a8, p.q, stage + line_off, lx, chunk0 + 2);
-                    release_aux();
-                } else {
-                    const int key = cw;
-                    if (MODE == MODE_BWDX || key != lut_key) {  // dX: every stage brings other rows
-                        float a[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            a[i] = (i < p.q) ? ptx::ld_shared_f32(aux + a_off + i * (kRows * 4)) * wscale : 0.0f;
-                        lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
-                        lut_key = key;
-                    }
-                    ok = acquire_slot();
-                    if (!ok) break;
-                    uint32_t S[4];
-                    selectors<NWC>(cv, S);
-                    expand32_codes<NWC>(S, lut, stage + line_off, lx, chunk0);
-                    release_aux();
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(ctl.aready + 8 * s);
-                advance(min(kPfGroups, iters - it));
-                if (MODE == MODE_FWD) {
-                    kpos += kPfGroups * kBlockK;
-                    while (kpos >= next_edge && cw < p.G - 1) { ++cw; next_edge += p.g; }
-                }
+        Cur cur;
+        cur.tile = (int)blockIdx.x;
+        cur.valid = cur.tile < num_tiles;
+        cur.fresh = true;
+        cur.it = group;
+        cur.iters = 0; cur.kb_begin = 0; cur.mt = 0; cur.c = 0; cur.kpos = 0; cur.next_edge = 0;
+        if (cur.valid) {
+            enter_tile(cur);
+            while (cur.it >= cur.iters) {
+                cur.it -= cur.iters;
+                cur.tile += gridDim.x;
+                if (cur.tile >= num_tiles) { cur.valid = false; break; }
+                enter_tile(cur);
             }
-            gi = (gi + iters) % kPfGroups;
+            if (cur.valid) locate(cur);
+        }
+        uint32_t cvA[NL], cvB[NL];
+        float avA[NS], avB[NS];
+        if (QM == QM_GENERIC) {
+            // q > 4: one set of registers, loaded at the head of the task (under the wait for the slot)
+            while (cur.valid && ok) {
+                issue(cur, cvA, avA);
+                ok = process(cur, cvA, avA);
+                advance(cur);
+            }
+        } else {
+            // q <= 4: the loads of the next task are in flight while this one is expanded (two
+            // register sets, so that nothing has to wait for a load in order to be moved)
+            if (cur.valid) issue(cur, cvA, avA);
+            while (cur.valid && ok) {
+                Cur nxt = cur;
+                advance(nxt);
+                if (nxt.valid) issue(nxt, cvB, avB);
+                ok = process(cur, cvA, avA);
+                cur = nxt;
+                if (!cur.valid || !ok) break;
+                advance(nxt);
+                if (nxt.valid) issue(nxt, cvA, avA);
+                ok = process(cur, cvB, avB);
+                cur = nxt;
+            }
         }
         if (p.helpers && ok && (int)blockIdx.x < num_tiles) {
             // share the epilogue of this CTA's last tile.  Its operand slots are free once the
@@ -929,7 +943,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 ptx::tc_fence_after_sync();
                 const int quarter = warp & 3, helper = 1 + (warp >> 2);  // 1..6
                 const int m0w = m0 + quarter * 32;
-                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
+                const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * kAccCols;
                 const uint32_t buf = smem_base + (uint32_t)warp * 1024u;
                 const float winv = 1.0f / wscale;  // a power of two
                 const int g = lane >> 2, tq = lane & 3;
@@ -977,7 +991,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             for (int i = et; i < TN; i += kPfEpiWarps * 32)
                 scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
             asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
-            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7);
+            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7, 512u);  // a whole tile away: poll rarely
             if (!ok) break;
             ptx::tc_fence_after_sync();
             // accumulator row `lane` of this warp's quarter is output column m0w + lrow
@@ -986,7 +1000,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const float bias = (MODE == MODE_FWD && p.bias != nullptr && p.splits == 1 && m0w + lrow < p.Mdim)
                                    ? __ldg(p.bias + m0w + lrow) : 0.0f;
             uint8_t* tile_out = out_base + ((p.splits > 1) ? (long long)z * p.n * p.Mdim * 4 : 0);
-            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * TmemCols<TN>::value;
+            const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * kAccCols;
             const bool full_rows = vec_ok && (m0w + 32 <= p.Mdim);
             if (p.fast_epi) {
                 const int g = lane >> 2, tq = lane & 3;
@@ -1385,14 +1399,15 @@ decode_kernel(const __grid_constant__ CUtensorMap tmap_bits, const DecodeParams 
 
 struct ExpandPlan {
     int TN, splits, kb_per_split, num_kb, m_tiles, n_tiles;
-    int stages, aux_slots, epi_bufs, alpha_parts;
-    uint32_t bits_bytes, alpha_bytes;
+    int a_slots, b_slots, epi_bufs;
+    uint32_t bits_bytes, alpha_bytes;                                    // one stage's chunk of the planes; the scales of one (row block, group)
     size_t planes_bytes;                                                 // the regrouped planes (codes for q <= 4)
     size_t smem;                                                         // dynamic shared memory of the GEMM kernel
     size_t off_tok, off_act, off_alpha, off_bits, off_partial, total;  // workspace layout (bytes)
     int ld_act;                                                          // pitch of the fp16 activations (elements)
 };
 
+constexpr int kPfMinWidth = 176;                                       // token-tile width below which the workers, not the UMMAs, set the pace
 constexpr size_t kSmemLimit = 232448;                                   // 227 KiB per CTA
 constexpr size_t kPfFixedBytes = 1024 + kPfCtlBytes + kPfScaleBytes;   // alignment slack, barriers, output scales
 
@@ -1411,7 +1426,20 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     if (n <= 32) tn = 32;
     else if (n <= 64) tn = 64;
     else if (n <= 128) tn = 128;
-    else tn = 256;  // the expansion and the UMMA issue cost the same per stage whatever the width
+    else {
+        // Any multiple of 16 up to 256 is a legal UMMA width.  The kernel is persistent with
+        // ceil(tiles / SMs) tiles per CTA, so its time goes with that count times the width (the
+        // UMMAs of a stage take time in proportion to it) -- except that below kPfMinWidth the
+        // workers, who expand one weight tile per stage whatever the width, set the pace.  The
+        // width that minimises the product wins; ties go to the wider tile (fewer expansions).
+        long long best = -1;
+        tn = 256;
+        for (int c = 256; c >= 128; c -= 16) {
+            const long long per_cta = ceil_div(pl.m_tiles * ceil_div(n, c), sms);
+            const long long cost = per_cta * (c > kPfMinWidth ? c : kPfMinWidth);
+            if (best < 0 || cost < best) { best = cost; tn = c; }
+        }
+    }
     pl.TN = tn;
     pl.n_tiles = ceil_div(n, tn);
     const int tiles = pl.m_tiles * pl.n_tiles;
@@ -1425,38 +1453,22 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     pl.kb_per_split = ceil_div(pl.num_kb, splits);
     pl.splits = ceil_div(pl.num_kb, pl.kb_per_split);
 
-    // one stage: A tile, B tile, the stage's plane words (q KiB), the scales of every group the
-    // stage's k range can touch, 16 bytes of group indices
     const int rows = (mode == MODE_FWD) ? 128 : 64;
-    const int kspan = (mode == MODE_FWD) ? 64 : 128;
-    pl.alpha_parts = (g % kspan == 0) ? 1 : ((g % (kspan / 2) == 0) ? 2 : 4);
-    if (mode == MODE_FWD && pl.alpha_parts == 4) pl.alpha_parts = 2;  // g % 32 == 0 always holds
     pl.bits_bytes = (q <= 3 ? 3u : (uint32_t)q) * 1024u;  // q <= 4: selector codes (3 or 4 words per 32 weights)
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
-    const size_t ab_bytes = kABytes + (size_t)tn * kBlockK * 2;
-    const size_t aux_bytes = pl.bits_bytes + (size_t)pl.alpha_parts * pl.alpha_bytes;
-    auto smem_of = [&](int stages, int aux_slots, int epi_bufs) {
-        return stages * ab_bytes + aux_slots * aux_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
+    // Shared memory: as many weight slots as there are worker groups (a group refills its slot as
+    // soon as the UMMAs that read it are done), the rest for the ring of activation tiles and a
+    // second staging buffer for the epilogue.
+    const size_t b_bytes = (size_t)tn * kBlockK * 2;
+    auto smem_of = [&](int a_slots, int b_slots, int epi_bufs) {
+        return a_slots * (size_t)kABytes + b_slots * b_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
     };
-    // operand slots first (a multiple of the number of worker groups, which take stages in turn:
-    // then a group meets the same slots in every round and never waits on a barrier phase it has
-    // not seen complete), then a longer ring of weight chunks and a second staging buffer for the
-    // epilogue as far as they fit
-    pl.stages = kPfGroups;
-    for (int st = (kPfMaxStages / kPfGroups) * kPfGroups; st >= kPfGroups; st -= kPfGroups)
-        if (smem_of(st, st, 1) <= kSmemLimit) { pl.stages = st; break; }
-    pl.aux_slots = pl.stages;
-    pl.epi_bufs = 1;
-    const int tries[5][2] = {{2 * kPfGroups, 2}, {kPfGroups, 2}, {2 * kPfGroups, 1}, {kPfGroups, 1}, {0, 2}};
-    for (int t = 0; t < 5; ++t) {
-        const int ax = pl.stages + tries[t][0];
-        if (ax <= kPfMaxStages && smem_of(pl.stages, ax, tries[t][1]) <= kSmemLimit) {
-            pl.aux_slots = ax;
-            pl.epi_bufs = tries[t][1];
-            break;
-        }
-    }
-    pl.smem = smem_of(pl.stages, pl.aux_slots, pl.epi_bufs);
+    pl.a_slots = kPfGroups;
+    pl.epi_bufs = 2;
+    pl.b_slots = 2;
+    for (int nb = kPfMaxSlots; nb >= 2; --nb)
+        if (smem_of(pl.a_slots, nb, pl.epi_bufs) <= kSmemLimit) { pl.b_slots = nb; break; }
+    pl.smem = smem_of(pl.a_slots, pl.b_slots, pl.epi_bufs);
 
     const size_t chunks_bits = (size_t)pl.m_tiles * pl.num_kb;                       // [m_tile][kb] or [u][jb]
     const size_t blocks_alpha = (size_t)((mode == MODE_FWD) ? pl.m_tiles : pl.num_kb) * G;  // [m_tile][G] or [jb][G]
@@ -1492,10 +1504,10 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
-template <int MODE, int TN, int QM>
+template <int MODE, int QM>
 bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
                          cudaStream_t stream) {
-    auto kern = expand_gemm_kernel<MODE, TN, QM>;
+    auto kern = expand_gemm_kernel<MODE, QM>;
     bcq_status st0 = ensure_dynamic_smem(kern, pl.smem);
     if (st0 != BCQ_OK) return st0;
     const int tiles = pl.m_tiles * pl.n_tiles * pl.splits;
@@ -1510,12 +1522,12 @@ bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const Ex
     return BCQ_OK;
 }
 
-template <int MODE, int TN>
+template <int MODE>
 bcq_status launch_expand_q(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
                            cudaStream_t stream) {
-    if (p.q <= 3) return launch_expand<MODE, TN, QM_LUT3>(tm, tmo, p, pl, stream);
-    if (p.q == 4) return launch_expand<MODE, TN, QM_LUT4>(tm, tmo, p, pl, stream);
-    return launch_expand<MODE, TN, QM_GENERIC>(tm, tmo, p, pl, stream);
+    if (p.q <= 3) return launch_expand<MODE, QM_LUT3>(tm, tmo, p, pl, stream);
+    if (p.q == 4) return launch_expand<MODE, QM_LUT4>(tm, tmo, p, pl, stream);
+    return launch_expand<MODE, QM_GENERIC>(tm, tmo, p, pl, stream);
 }
 
 // act: bf16 [n][ldact] with Kdim valid columns (X for the forward, dY for dX).
@@ -1601,8 +1613,10 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.pitch = pitch;
     p.n = n; p.Mdim = Mdim; p.num_kb = pl.num_kb; p.kb_per_split = pl.kb_per_split; p.splits = pl.splits;
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
-    p.stages = pl.stages; p.aux_slots = pl.aux_slots; p.epi_bufs = pl.epi_bufs; p.bits_bytes = pl.bits_bytes;
-    p.alpha_bytes = pl.alpha_bytes; p.alpha_parts = pl.alpha_parts;
+    p.tn = pl.TN;
+    p.acc_cols = 32;
+    while ((int)p.acc_cols < pl.TN) p.acc_cols *= 2;
+    p.a_slots = pl.a_slots; p.b_slots = pl.b_slots; p.epi_bufs = pl.epi_bufs; p.chunk_words = pl.bits_bytes / 4;
     p.bits_t = (coded && prepared != nullptr) ? reinterpret_cast<const uint32_t*>(prepared) : pp.bits_t;
     p.alpha_t = pp.alpha_t; p.bias = bias; p.hdr = hdr; p.tok_inv_scale = tok;
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
@@ -1615,16 +1629,11 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
         if (st != BCQ_OK) return st;
     }
     // The workers find the last tile's accumulator by barrier parity alone.  They run at most
-    // `stages` pipeline stages ahead of the tensor core, so the parity is unambiguous only if
+    // `a_slots` pipeline stages ahead of the tensor core, so the parity is unambiguous only if
     // two tiles are longer than that: then the accumulator's previous use (two tiles back) is
     // certain to be complete when a worker has finished the last tile's stages.
-    p.helpers = (p.fast_epi && 2 * pl.num_kb >= pl.stages + 2) ? 1 : 0;
-    switch (pl.TN) {
-        case 32: st = launch_expand_q<MODE, 32>(tm, tmo, p, pl, s); break;
-        case 64: st = launch_expand_q<MODE, 64>(tm, tmo, p, pl, s); break;
-        case 128: st = launch_expand_q<MODE, 128>(tm, tmo, p, pl, s); break;
-        default: st = launch_expand_q<MODE, 256>(tm, tmo, p, pl, s); break;
-    }
+    p.helpers = (p.fast_epi && 2 * pl.num_kb >= pl.a_slots + 2) ? 1 : 0;
+    st = launch_expand_q<MODE>(tm, tmo, p, pl, s);
     if (st != BCQ_OK) return st;
     if (pl.splits > 1) {
         const long long total = (long long)n * Mdim;
