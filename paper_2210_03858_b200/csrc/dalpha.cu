@@ -141,27 +141,29 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // the whole warp walks the loop (uniform control flow), one elected lane issues
-        bool ok = true;
-        int s = 0, lt = 0;
-        uint32_t ph = 0;
-        // descriptor halves (128-byte swizzle, MN-major: leading offset 8192 B between blocks of 64
-        // rows, stride 1024 B between groups of eight token lines); a UMMA steps the start by 2048 B
-        constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);
-        constexpr uint32_t kLoExtra = (8192u >> 4) << 16;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
-            int j0, k0, z, kb_begin, iters;
-            tile_coords(tile, j0, k0, z, kb_begin, iters);
-            const int acc = lt & 1;
-            ok = wait_bar(acc_empty + 8 * acc, (uint32_t)((lt >> 1) & 1) ^ 1u, ctl, 17);
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
-            for (int it = 0; it < iters; ++it) {
-                ok = wait_bar(ctl.full + 8 * s, ph, ctl, 13);
+        // One elected thread runs the whole loop: between two stages it has a barrier check, a
+        // fence, four UMMAs and a commit to get through in less time than the tensor core needs
+        // for a stage, so nothing warp-wide (election, reconvergence) is left inside the loop.
+        if (ptx::elect_one()) {
+            bool ok = true;
+            int s = 0, lt = 0;
+            uint32_t ph = 0;
+            // descriptor halves (128-byte swizzle, MN-major: leading offset 8192 B between blocks of 64
+            // rows, stride 1024 B between groups of eight token lines); a UMMA steps the start by 2048 B
+            constexpr uint32_t kHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+            constexpr uint32_t kLoExtra = (8192u >> 4) << 16;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+                int j0, k0, z, kb_begin, iters;
+                tile_coords(tile, j0, k0, z, kb_begin, iters);
+                const int acc = lt & 1;
+                ok = wait_bar(acc_empty + 8 * acc, (uint32_t)((lt >> 1) & 1) ^ 1u, ctl, 17);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                if (ptx::elect_one()) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
+                for (int it = 0; it < iters; ++it) {
+                    ok = wait_bar(ctl.full + 8 * s, ph, ctl, 13, 32u);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
                     const uint32_t a_lo = (((smem_base + (uint32_t)s * kStageBytes) >> 4) & 0x3FFFu) | kLoExtra;
                     const uint32_t b_lo = a_lo + (kABytes >> 4);
 #pragma unroll
@@ -169,18 +171,16 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
                         ptx::umma_f16_halves(d_tmem, a_lo + kk * (2048u >> 4), kHi, b_lo + kk * (2048u >> 4), kHi, kIdesc,
                                              (it > 0 || kk > 0) ? 1u : 0u);
                     ptx::umma_commit(ctl.empty + 8 * s);
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
-                __syncwarp();
-                if (++s == STAGES) { s = 0; ph ^= 1u; }
+                if (ok) ptx::umma_commit(ctl.accum + 8 * acc);
             }
-            if (ok && ptx::elect_one()) ptx::umma_commit(ctl.accum + 8 * acc);
-            __syncwarp();
+            if (!ok) {
+                ptx::umma_commit(ctl.spare);
+                wait_bar(ctl.spare, 0, ctl, 15);
+            }
         }
-        if (!ok) {
-            if (ptx::elect_one()) ptx::umma_commit(ctl.spare);
-            __syncwarp();
-            wait_bar(ctl.spare, 0, ctl, 15);
-        }
+        __syncwarp();
     } else {
         // ---------------- epilogue: thread = (row j, HN columns of the tile)
         const int quarter = warp & 3;

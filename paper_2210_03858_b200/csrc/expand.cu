@@ -521,28 +521,28 @@ struct StageLayout {
 
 // Prefill kernel.  Persistent: every CTA walks over output tiles (m-tile fastest, so that CTAs
 // running at the same time share activation tiles in L2).  32 warps:
-//   warps 0..23   workers in three groups of eight; group g takes the pipeline stages whose running
-//                 index is g mod 3.  A thread expands 32 weights of one row per stage, so a group
-//                 rebuilds one 128 x 64 weight tile.  The thread reads its selector codes (or plane
-//                 words) and scales straight from the regrouped arrays in global memory, one task
-//                 ahead of the one it expands, so the loads are hidden behind a whole turn of the
-//                 group
-//   warp 24       UMMA issuer, owner of the tensor-memory allocation (two accumulators)
-//   warp 25       producer of the activation tiles (TMA)
-//   warps 28..31  epilogue: drain one accumulator while the main loop fills the other (warp w
+//   warps 0..11   workers in three groups of four; group g takes the pipeline stages whose running
+//                 index is g mod 3.  A thread expands 64 weights of one row per stage (one 128-byte
+//                 line of the operand tile), so a group rebuilds one 128 x 64 weight tile.  The
+//                 thread reads its selector codes (or plane words) and scales straight from the
+//                 regrouped arrays in global memory, one task ahead of the one it expands, so the
+//                 loads are hidden behind a whole turn of the group
+//   warp 12       UMMA issuer, owner of the tensor-memory allocation (two accumulators)
+//   warp 13       producer of the activation tiles (TMA)
+//   warps 16..19  epilogue: drain one accumulator while the main loop fills the other (warp w
 //                 reaches the tensor-memory lanes 32 * (w % 4) .. + 31)
 // Shared memory: a ring of weight tiles (16 KiB each; few, the workers refill one as soon as the
 // tensor core is done with it), a deeper ring of activation tiles (TN x 128 B each; a TMA load
 // takes about a microsecond to land), the epilogue's staging, barriers and output scales.
 constexpr int kPfGroups = 3;
-constexpr int kPfGroupWarps = 8;
-constexpr int kPfWorkerWarps = kPfGroups * kPfGroupWarps;  // 24
-constexpr int kPfMmaWarp = kPfWorkerWarps;                 // 24
-constexpr int kPfProdWarp = kPfMmaWarp + 1;                // 25
-constexpr int kPfEpiWarp0 = 28;
+constexpr int kPfGroupWarps = 4;
+constexpr int kPfWorkerWarps = kPfGroups * kPfGroupWarps;  // 12
+constexpr int kPfMmaWarp = kPfWorkerWarps;                 // 12
+constexpr int kPfProdWarp = kPfMmaWarp + 1;                // 13
+constexpr int kPfEpiWarp0 = 16;
 constexpr int kPfEpiWarps = 4;
-constexpr int kPfWarps = kPfEpiWarp0 + kPfEpiWarps;        // 32
-constexpr int kPfThreads = kPfWarps * 32;                  // 1024
+constexpr int kPfWarps = kPfEpiWarp0 + kPfEpiWarps;        // 20
+constexpr int kPfThreads = kPfWarps * 32;                  // 640
 static_assert(kPfEpiWarp0 % 4 == 0, "epilogue warp e must sit on tensor-memory lane quarter e");
 __device__ __forceinline__ int pf_worker_index(int warp) { return warp < kPfWorkerWarps ? warp : -1; }
 __device__ __forceinline__ int pf_epilogue_index(int warp) { return warp >= kPfEpiWarp0 ? warp - kPfEpiWarp0 : -1; }
@@ -669,9 +669,9 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         }
     };
     // On the last tile of a CTA the worker warps have nothing left to expand, so they share its
-    // epilogue: of the seven warps on a tensor-memory lane quarter (one epilogue warp, six workers)
-    // warp h takes the boxes h, h + 7, ...
-    constexpr int kPfHelpers = 1 + kPfWorkerWarps / 4;  // 7
+    // epilogue: of the four warps on a tensor-memory lane quarter (one epilogue warp, three workers)
+    // warp h takes the boxes h, h + 4, ...
+    constexpr int kPfHelpers = 1 + kPfWorkerWarps / 4;  // 4
     auto is_last_tile = [&](int tile) { return tile + (int)gridDim.x >= num_tiles; };
 
     if (warp == kPfProdWarp) {
@@ -685,7 +685,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 int m0, t0, z, kb_begin, iters;
                 tile_coords(tile, m0, t0, z, kb_begin, iters);
                 for (int it = 0; it < iters; ++it) {
-                    ok = wait_bar(b_empty + 8 * s, ph ^ 1u, ctl, 1);
+                    ok = wait_bar(b_empty + 8 * s, ph ^ 1u, ctl, 1, 256u);
                     if (!ok) break;
                     const uint32_t bar = ctl.full + 8 * s;
                     ptx::mbar_arrive_expect_tx(bar, kBBytes);
@@ -707,34 +707,41 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             }
         }
     } else if (warp == kPfMmaWarp) {
-        // ---------------- UMMA issuer: the whole warp walks the stages and waits on the barriers
-        // (warp-uniform control flow); one elected lane issues
-        bool ok = true;
-        int sa = 0, sb = 0, lt = 0;
-        uint32_t pha = 0, phb = 0;
-        // shared-memory descriptor halves (128-byte swizzle, version 1): low = start address >> 4 and
-        // leading offset >> 4 at bit 16, high = stride offset >> 4, version at bit 14, swizzle at bit 29
-        constexpr uint32_t kHiCommon = (1024u >> 4) | (1u << 14) | (2u << 29);
-        constexpr uint32_t kAHi = kHiCommon, kBHi = kHiCommon;
-        constexpr uint32_t kALoExtra = ((MODE == MODE_FWD) ? (16u >> 4) : (8192u >> 4)) << 16;  // leading offset of A
-        constexpr uint32_t kBLoExtra = (16u >> 4) << 16;
-        constexpr uint32_t kAStep = (MODE == MODE_FWD) ? (32u >> 4) : (2048u >> 4);
-        const uint32_t a_lo0 = ((smem_base >> 4) & 0x3FFFu) | kALoExtra;
-        const uint32_t b_lo0 = ((b_base >> 4) & 0x3FFFu) | kBLoExtra;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
-            int m0, t0, z, kb_begin, iters;
-            tile_coords(tile, m0, t0, z, kb_begin, iters);
-            const int acc = lt & 1;
-            const uint32_t acc_ph = (lt >> 1) & 1;
-            ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
-            if (!ok) break;
-            ptx::tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
-            for (int it = 0; it < iters; ++it) {
-                ok = wait_bar(ctl.full + 8 * sb, phb, ctl, 4, 32u) && wait_bar(ctl.aready + 8 * sa, pha, ctl, 3, 32u);
+        // ---------------- UMMA issuer.  One elected thread runs the whole loop: per stage it has
+        // to get through two barrier checks, a fence, four UMMAs and two commits in less time
+        // than the tensor core needs for the stage (512 cycles at the full width), so nothing
+        // warp-wide (election, reconvergence) is left inside the loop and the two barrier checks
+        // are issued together.
+        if (ptx::elect_one()) {
+            bool ok = true;
+            int sa = 0, sb = 0, lt = 0;
+            uint32_t pha = 0, phb = 0;
+            // shared-memory descriptor halves (128-byte swizzle, version 1): low = start address >> 4 and
+            // leading offset >> 4 at bit 16, high = stride offset >> 4, version at bit 14, swizzle at bit 29
+            constexpr uint32_t kHiCommon = (1024u >> 4) | (1u << 14) | (2u << 29);
+            constexpr uint32_t kAHi = kHiCommon, kBHi = kHiCommon;
+            constexpr uint32_t kALoExtra = ((MODE == MODE_FWD) ? (16u >> 4) : (8192u >> 4)) << 16;  // leading offset of A
+            constexpr uint32_t kBLoExtra = (16u >> 4) << 16;
+            constexpr uint32_t kAStep = (MODE == MODE_FWD) ? (32u >> 4) : (2048u >> 4);
+            const uint32_t a_lo0 = ((smem_base >> 4) & 0x3FFFu) | kALoExtra;
+            const uint32_t b_lo0 = ((b_base >> 4) & 0x3FFFu) | kBLoExtra;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+                int m0, t0, z, kb_begin, iters;
+                tile_coords(tile, m0, t0, z, kb_begin, iters);
+                const int acc = lt & 1;
+                const uint32_t acc_ph = (lt >> 1) & 1;
+                ok = wait_bar(acc_empty + 8 * acc, acc_ph ^ 1u, ctl, 8);  // the epilogue has drained it
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                if (ptx::elect_one()) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
+                for (int it = 0; it < iters; ++it) {
+                    // both operands of the stage in place?  (the common case: yes, both at once)
+                    const bool fb = ptx::mbar_try_wait(ctl.full + 8 * sb, phb);
+                    const bool fa = ptx::mbar_try_wait(ctl.aready + 8 * sa, pha);
+                    if (!fb) ok = wait_bar(ctl.full + 8 * sb, phb, ctl, 4, 32u);
+                    if (!fa && ok) ok = wait_bar(ctl.aready + 8 * sa, pha, ctl, 3, 32u);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
                     // descriptors: only the start-address field changes, by 32 bytes (K-major) or
                     // 2048 bytes (MN-major A) per UMMA
                     const uint32_t a_lo = a_lo0 + (uint32_t)sa * (kABytes >> 4);
@@ -745,41 +752,41 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                                              (it > 0 || kk > 0) ? 1u : 0u);
                     ptx::umma_commit(ctl.empty + 8 * sa);
                     ptx::umma_commit(b_empty + 8 * sb);
+                    if (++sa == NA) { sa = 0; pha ^= 1u; }
+                    if (++sb == NB) { sb = 0; phb ^= 1u; }
                 }
-                __syncwarp();
-                if (++sa == NA) { sa = 0; pha ^= 1u; }
-                if (++sb == NB) { sb = 0; phb ^= 1u; }
+                if (ok) ptx::umma_commit(ctl.accum + 8 * acc);
             }
-            if (ok && ptx::elect_one()) ptx::umma_commit(ctl.accum + 8 * acc);
-            __syncwarp();
+            if (!ok) {
+                ptx::umma_commit(ctl.spare);
+                wait_bar(ctl.spare, 0, ctl, 5);
+            }
         }
-        if (!ok) {
-            if (ptx::elect_one()) ptx::umma_commit(ctl.spare);
-            __syncwarp();
-            wait_bar(ctl.spare, 0, ctl, 5);
-        }
+        __syncwarp();
     } else if (pf_worker_index(warp) >= 0) {
         // ---------------- workers
-        const int wid = pf_worker_index(warp);  // 0..23
-        const int group = wid >> 3;           // takes the stages whose running index is `group` mod kPfGroups
-        const int wl = wid & 7;
+        const int wid = pf_worker_index(warp);  // 0..11
+        const int group = wid / kPfGroupWarps;  // takes the stages whose running index is `group` mod kPfGroups
+        const int wl = wid % kPfGroupWarps;
         const float wscale = pow2f(weight_shift(p.hdr, p.q));
 
-        // fwd : task = (weight row m0 + row, 32-wide half of the stage's 64 k); the two halves of a
-        //       row sit in adjacent lanes
-        // dX  : task = (K index j = 64*kb + row, 32-wide quarter of the tile's 128 k); the four
-        //       quarters of a row sit in adjacent lanes
-        const int row = (MODE == MODE_FWD) ? wl * 16 + (lane >> 1) : wl * 8 + (lane >> 2);
-        const int part = (MODE == MODE_FWD) ? (lane & 1) : (lane & 3);
-        const uint32_t line_off = (MODE == MODE_FWD) ? row * 128 : ((part >> 1) * 8192) + row * 128;
+        // A task is one 128-byte line of the weight tile: 64 weights of one row.
+        // fwd : (weight row m0 + row, the stage's 64 k); a warp takes 32 consecutive rows
+        // dX  : (K index j = 64*kb + row, 64-wide half of the tile's 128 k); the two halves of a row
+        //       sit in adjacent lanes
+        // Either way the 32 lanes of a warp write their 16-byte chunks to all banks evenly.
+        const int row = (MODE == MODE_FWD) ? wl * 32 + lane : wl * 16 + (lane >> 1);
+        const int half = (MODE == MODE_FWD) ? 0 : (lane & 1);
+        const uint32_t line_off = (uint32_t)half * 8192u + (uint32_t)row * 128u;
         const uint32_t lx = row & 7;
-        const uint32_t chunk0 = (MODE == MODE_FWD) ? part * 4 : (part & 1) * 4;
         constexpr int NWC = CodeWords<QM>::value;
-        constexpr int NL = (QM == QM_GENERIC) ? NW : NWC;   // words a task loads
+        constexpr int NL = (QM == QM_GENERIC) ? NW : NWC;   // words a 32-weight block loads
         constexpr int NS = (QM == QM_GENERIC) ? NW : 4;     // scales a task loads
         // the task's words within a chunk [m_tile][kb] (fwd) or [u][jb] (dX) of the regrouped planes:
-        // q <= 4 selector codes [row][block][NWC], q > 4 plane words [plane][row][block]
-        const uint32_t word_off = (QM == QM_GENERIC) ? (uint32_t)(row * kUnit + part) : (uint32_t)((row * kUnit + part) * NWC);
+        // q <= 4 selector codes [row][block][NWC], q > 4 plane words [plane][row][block]; its two
+        // 32-weight blocks are neighbours
+        const uint32_t block0 = (uint32_t)(row * kUnit + half * 2);
+        const uint32_t word_off = (QM == QM_GENERIC) ? block0 : block0 * NWC;
         const uint32_t chunk_words = p.chunk_words;
         const uint32_t alpha_block = (uint32_t)p.q * kRows;  // floats per (row block, group): [plane][row]
 
@@ -787,7 +794,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // is `group` mod kPfGroups.  A cursor names one of them.
         struct Cur {
             int tile, it, iters, kb_begin, mt;
-            int c, kpos, next_edge;  // group index of the task's 32 k (forward: advances with the stage)
+            int c, kpos, next_edge;  // group index of the task's first 32 k (forward: advances with the stage)
+            bool split;              // the second 32 k belong to the next group (g not a multiple of 64)
             bool fresh;              // the scales differ from the previous task's: load them, rebuild the table
             bool valid;
         };
@@ -797,9 +805,10 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             x.mt = m0 >> 7;
         };
         auto locate = [&](Cur& x) {  // group index at (tile, it), from scratch
-            x.kpos = (MODE == MODE_FWD) ? (x.kb_begin + x.it) * kBlockK + part * 32 : x.mt * kBlockM + part * 32;
+            x.kpos = (MODE == MODE_FWD) ? (x.kb_begin + x.it) * kBlockK : x.mt * kBlockM + half * 64;
             x.c = min(x.kpos / p.g, p.G - 1);
             x.next_edge = (x.c + 1) * p.g;
+            x.split = (x.kpos + 32 >= x.next_edge) && (x.c < p.G - 1);
         };
         // to the next task: kPfGroups stages on
         auto advance = [&](Cur& x) {
@@ -819,27 +828,41 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 const int c0 = x.c;
                 x.kpos += kPfGroups * kBlockK;
                 while (x.kpos >= x.next_edge && x.c < p.G - 1) { ++x.c; x.next_edge += p.g; }
-                x.fresh = (QM == QM_GENERIC) || (x.c != c0);
+                x.split = (x.kpos + 32 >= x.next_edge) && (x.c < p.G - 1);
+                x.fresh = (QM == QM_GENERIC) || (x.c != c0) || x.split;
             } else {
                 x.fresh = true;  // dX: every stage brings other rows
             }
         };
+        auto alpha_ptr = [&](const Cur& x, int c) {
+            const int blk = (MODE == MODE_FWD) ? x.mt : x.kb_begin + x.it;
+            return p.alpha_t + ((long long)blk * p.G + c) * alpha_block + row;
+        };
         // global loads of a task: its plane words or codes and, when they change, its scales
-        auto issue = [&](const Cur& x, uint32_t (&cv)[NL], float (&av)[NS]) {
+        auto issue = [&](const Cur& x, uint32_t (&cv)[2][NL], float (&av)[NS]) {
             const uint32_t* src = p.bits_t + ((long long)x.mt * p.num_kb + x.kb_begin + x.it) * chunk_words + word_off;
             if (QM == QM_GENERIC) {
 #pragma unroll
-                for (int i = 0; i < NL; ++i) cv[i] = (i < p.q) ? ptx::ldg_nc_u32(src + i * (kRows * kUnit)) : 0u;
+                for (int i = 0; i < NL; ++i) {
+                    if (i < p.q) {
+                        const uint2 v = ptx::ldg_nc_v2(src + i * (kRows * kUnit));
+                        cv[0][i] = v.x; cv[1][i] = v.y;
+                    } else {
+                        cv[0][i] = 0u; cv[1][i] = 0u;
+                    }
+                }
             } else if (NWC == 4) {
-                const uint4 v = ptx::ldg_nc_v4(src);
-                cv[0] = v.x; cv[1] = v.y; cv[2] = v.z; cv[NL - 1] = v.w;
+                const uint4 v0 = ptx::ldg_nc_v4(src), v1 = ptx::ldg_nc_v4(src + 4);
+                cv[0][0] = v0.x; cv[0][1] = v0.y; cv[0][2] = v0.z; cv[0][NL - 1] = v0.w;
+                cv[1][0] = v1.x; cv[1][1] = v1.y; cv[1][2] = v1.z; cv[1][NL - 1] = v1.w;
             } else {
-#pragma unroll
-                for (int i = 0; i < NL; ++i) cv[i] = ptx::ldg_nc_u32(src + i);
+                // six words, 8-byte aligned
+                const uint2 v0 = ptx::ldg_nc_v2(src), v1 = ptx::ldg_nc_v2(src + 2), v2 = ptx::ldg_nc_v2(src + 4);
+                cv[0][0] = v0.x; cv[0][1] = v0.y; cv[0][2] = v1.x;
+                cv[1][0] = v1.y; cv[1][1] = v2.x; cv[1][2] = v2.y;
             }
             if (x.fresh) {
-                const int blk = (MODE == MODE_FWD) ? x.mt : x.kb_begin + x.it;
-                const float* ap = p.alpha_t + ((long long)blk * p.G + x.c) * alpha_block + row;
+                const float* ap = alpha_ptr(x, x.c);
 #pragma unroll
                 for (int i = 0; i < NS; ++i)
                     av[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
@@ -848,37 +871,51 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
 
         Lut lut = {0u, 0u, 0u, 0u};
         bool ok = true;
-        int s = group;  // weight slot of the current task (NA >= kPfGroups)
+        int s = group;  // weight slot of the current task (a_slots >= kPfGroups)
         uint32_t ph = 0;
         // One task: wait until the UMMAs that read the slot's previous contents are done (the first
         // warp of the group polls the barrier, the others park on a hardware barrier: a polling
         // warp takes issue slots from the warps that expand), expand, publish.
-        auto process = [&](const Cur& x, const uint32_t (&cv)[NL], const float (&av)[NS]) -> bool {
-            if (wl == 0) wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9, 32u);  // a timeout shows in the abort flag
+        auto process = [&](const Cur& x, const uint32_t (&cv)[2][NL], const float (&av)[NS]) -> bool {
+            if (wl == 0) wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9, 256u);  // a timeout shows in the abort flag
             ptx::named_bar_sync(kPfGroupBar0 + group, kPfGroupWarps * 32);
             if (*ctl.abort_flag) return false;
             const uint32_t line = smem_base + (uint32_t)s * kABytes + line_off;
-            if (QM == QM_GENERIC) {
-                float a8[BCQ_MAX_Q];
-                uint32_t w8[BCQ_MAX_Q];
+            float a2[NS];  // scales of the second 32 weights when they belong to the next group
+            if (x.split) {
+                const float* ap = alpha_ptr(x, x.c + 1);
 #pragma unroll
-                for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                    a8[i] = av[i % NS] * wscale;
-                    w8[i] = cv[i % NL];
+                for (int i = 0; i < NS; ++i)
+                    a2[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
+            }
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                const bool second = (b == 1) && x.split;
+                if (QM == QM_GENERIC) {
+                    float a8[BCQ_MAX_Q];
+                    uint32_t w8[BCQ_MAX_Q];
+#pragma unroll
+                    for (int i = 0; i < BCQ_MAX_Q; ++i) {
+                        a8[i] = (second ? a2[i % NS] : av[i % NS]) * wscale;
+                        w8[i] = cv[b][i % NL];
+                    }
+                    expand16_sum(w8, a8, p.q, line, lx, 4 * b);
+#pragma unroll
+                    for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
+                    expand16_sum(w8, a8, p.q, line, lx, 4 * b + 2);
+                } else {
+                    if ((b == 0 && x.fresh) || second) {
+                        float a[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) a[i] = (second ? a2[i % NS] : av[i % NS]) * wscale;
+                        lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
+                    }
+                    uint32_t cw[NWC], S[4];
+#pragma unroll
+                    for (int i = 0; i < NWC; ++i) cw[i] = cv[b][i % NL];
+                    selectors<NWC>(cw, S);
+                    expand32_codes<NWC>(S, lut, line, lx, 4 * b);
                 }
-                expand16_sum(w8, a8, p.q, line, lx, chunk0);
-#pragma unroll
-                for (int i = 0; i < BCQ_MAX_Q; ++i) w8[i] >>= 16;
-                expand16_sum(w8, a8, p.q, line, lx, chunk0 + 2);
-            } else {
-                if (x.fresh)
-                    lut = (QM == QM_LUT4) ? build_lut(av[0] * wscale, av[1] * wscale, av[2] * wscale, av[3 % NS] * wscale)
-                                          : build_lut(av[0] * wscale, av[1] * wscale, av[2] * wscale, 0.0f);
-                uint32_t cw[NWC], S[4];
-#pragma unroll
-                for (int i = 0; i < NWC; ++i) cw[i] = cv[i % NL];
-                selectors<NWC>(cw, S);
-                expand32_codes<NWC>(S, lut, line, lx, chunk0);
             }
             ptx::fence_proxy_async_smem();
             __syncwarp();
@@ -892,6 +929,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         cur.tile = (int)blockIdx.x;
         cur.valid = cur.tile < num_tiles;
         cur.fresh = true;
+        cur.split = false;
         cur.it = group;
         cur.iters = 0; cur.kb_begin = 0; cur.mt = 0; cur.c = 0; cur.kpos = 0; cur.next_edge = 0;
         if (cur.valid) {
@@ -904,7 +942,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             }
             if (cur.valid) locate(cur);
         }
-        uint32_t cvA[NL], cvB[NL];
+        uint32_t cvA[2][NL], cvB[2][NL];
         float avA[NS], avB[NS];
         if (QM == QM_GENERIC) {
             // q > 4: one set of registers, loaded at the head of the task (under the wait for the slot)
@@ -941,7 +979,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             ok = wait_bar(ctl.accum + 8 * acc, (uint32_t)(lt >> 1) & 1u, ctl, 10);
             if (ok) {
                 ptx::tc_fence_after_sync();
-                const int quarter = warp & 3, helper = 1 + (warp >> 2);  // 1..6
+                const int quarter = warp & 3, helper = 1 + (warp >> 2);  // 1..3
                 const int m0w = m0 + quarter * 32;
                 const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)acc * kAccCols;
                 const uint32_t buf = smem_base + (uint32_t)warp * 1024u;
@@ -991,7 +1029,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             for (int i = et; i < TN; i += kPfEpiWarps * 32)
                 scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
             asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
-            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7, 512u);  // a whole tile away: poll rarely
+            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7, 1000u);  // a whole tile away: poll rarely
             if (!ok) break;
             ptx::tc_fence_after_sync();
             // accumulator row `lane` of this warp's quarter is output column m0w + lrow
@@ -1456,18 +1494,23 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     const int rows = (mode == MODE_FWD) ? 128 : 64;
     pl.bits_bytes = (q <= 3 ? 3u : (uint32_t)q) * 1024u;  // q <= 4: selector codes (3 or 4 words per 32 weights)
     pl.alpha_bytes = (uint32_t)(q * rows * 4);
-    // Shared memory: as many weight slots as there are worker groups (a group refills its slot as
-    // soon as the UMMAs that read it are done), the rest for the ring of activation tiles and a
-    // second staging buffer for the epilogue.
+    // Shared memory.  A worker group takes a few hundred nanoseconds from "the tensor core is done
+    // with my slot" to "the slot holds the next tile", and a TMA load about a microsecond to land;
+    // both rings must be deep enough to cover that at one stage per ~0.3 us.  First choice that fits:
     const size_t b_bytes = (size_t)tn * kBlockK * 2;
     auto smem_of = [&](int a_slots, int b_slots, int epi_bufs) {
         return a_slots * (size_t)kABytes + b_slots * b_bytes + epi_bufs * (size_t)kPfStagingBuf + kPfFixedBytes;
     };
-    pl.a_slots = kPfGroups;
+    const int rings[8][2] = {{6, 5}, {5, 5}, {6, 4}, {5, 4}, {4, 4}, {4, 3}, {3, 3}, {3, 2}};
     pl.epi_bufs = 2;
+    pl.a_slots = kPfGroups;
     pl.b_slots = 2;
-    for (int nb = kPfMaxSlots; nb >= 2; --nb)
-        if (smem_of(pl.a_slots, nb, pl.epi_bufs) <= kSmemLimit) { pl.b_slots = nb; break; }
+    for (int r = 0; r < 8; ++r)
+        if (smem_of(rings[r][0], rings[r][1], pl.epi_bufs) <= kSmemLimit) {
+            pl.a_slots = rings[r][0];
+            pl.b_slots = rings[r][1];
+            break;
+        }
     pl.smem = smem_of(pl.a_slots, pl.b_slots, pl.epi_bufs);
 
     const size_t chunks_bits = (size_t)pl.m_tiles * pl.num_kb;                       // [m_tile][kb] or [u][jb]
