@@ -7,7 +7,9 @@
 // its accumulator row from tensor memory 32 columns at a time, applies the signs of every
 // requested plane from one 32-bit word of the packed planes, and sums per group.  Partial sums
 // (one per split over tokens, column sub-tile and group piece) go to the workspace and a second
-// kernel adds them in a fixed order, so the result does not depend on scheduling.
+// kernel adds them in a fixed order, so the result does not depend on scheduling.  When every
+// output has exactly one partial (no token split and a group per column sub-tile, e.g. g = 128)
+// the epilogue writes dalpha itself and the second kernel is not launched.
 #include "gemm_common.cuh"
 
 namespace {
@@ -27,6 +29,11 @@ struct DalphaParams {
     uint32_t plane_mask;
     const uint32_t* bits;
     float* partial;      // [splits][n_subtiles][q][slots][d_out]
+    // direct != 0: every output has exactly one partial (no token split, one group per column
+    // sub-tile), so the epilogue writes dalpha itself and no second kernel runs
+    int direct, accumulate;
+    float scale;
+    float* dalpha;       // [q][d_out][G]
 };
 
 
@@ -224,9 +231,14 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) {
                         if (i < p.q && ((p.plane_mask >> i) & 1u)) {
-                            const long long idx =
-                                ((((long long)z * p.n_subtiles + subtile) * p.q + i) * p.slots + slot) * p.d_out + j;
-                            p.partial[idx] = accs[i];
+                            if (p.direct) {
+                                float* dst = p.dalpha + ((long long)i * p.d_out + j) * p.G + c;
+                                *dst = p.accumulate ? (*dst + p.scale * accs[i]) : (p.scale * accs[i]);
+                            } else {
+                                const long long idx =
+                                    ((((long long)z * p.n_subtiles + subtile) * p.q + i) * p.slots + slot) * p.d_out + j;
+                                p.partial[idx] = accs[i];
+                            }
                         }
                     }
                 };
@@ -408,6 +420,8 @@ extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, in
     p.m_tiles = pl.m_tiles; p.n_tiles = pl.n_tiles;
     p.n_subtiles = pl.n_subtiles; p.slots = pl.slots; p.plane_mask = plane_mask;
     p.bits = bits; p.partial = reinterpret_cast<float*>(ws);
+    p.direct = (pl.splits == 1 && g == pl.HN) ? 1 : 0;
+    p.accumulate = accumulate; p.scale = scale; p.dalpha = dalpha;
     cudaStream_t s = (cudaStream_t)stream;
     // persistent, one CTA per SM; every CTA gets the same number of tiles (as many as the busiest
     // would get anyway), which leaves whole SMs to other kernels instead of a ragged last wave
@@ -425,6 +439,7 @@ extern "C" bcq_status bcq_linear_bwd_alpha(int d_out, int d_in, int q, int g, in
     }
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
+    if (p.direct) return BCQ_OK;
     const long long rblocks = (long long)q * p.G * ((d_out + 31) / 32);
     dalpha_reduce_kernel<<<(unsigned)rblocks, 256, 0, s>>>(
         d_out, d_in, q, g, p.G, pl.HN, pl.splits, pl.n_subtiles, pl.slots, plane_mask, scale, accumulate,

@@ -781,7 +781,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         const uint32_t lx = row & 7;
         constexpr int NWC = CodeWords<QM>::value;
         constexpr int NL = (QM == QM_GENERIC) ? NW : NWC;   // words a 32-weight block loads
-        constexpr int NS = (QM == QM_GENERIC) ? NW : 4;     // scales a task loads
+        constexpr int NSC = (QM == QM_GENERIC) ? NW : 4;    // scales a task loads
         // the task's words within a chunk [m_tile][kb] (fwd) or [u][jb] (dX) of the regrouped planes:
         // q <= 4 selector codes [row][block][NWC], q > 4 plane words [plane][row][block]; its two
         // 32-weight blocks are neighbours
@@ -839,7 +839,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             return p.alpha_t + ((long long)blk * p.G + c) * alpha_block + row;
         };
         // global loads of a task: its plane words or codes and, when they change, its scales
-        auto issue = [&](const Cur& x, uint32_t (&cv)[2][NL], float (&av)[NS]) {
+        auto issue = [&](const Cur& x, uint32_t (&cv)[2][NL], float (&av)[NSC]) {
             const uint32_t* src = p.bits_t + ((long long)x.mt * p.num_kb + x.kb_begin + x.it) * chunk_words + word_off;
             if (QM == QM_GENERIC) {
 #pragma unroll
@@ -864,7 +864,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             if (x.fresh) {
                 const float* ap = alpha_ptr(x, x.c);
 #pragma unroll
-                for (int i = 0; i < NS; ++i)
+                for (int i = 0; i < NSC; ++i)
                     av[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
             }
         };
@@ -876,16 +876,16 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         // One task: wait until the UMMAs that read the slot's previous contents are done (the first
         // warp of the group polls the barrier, the others park on a hardware barrier: a polling
         // warp takes issue slots from the warps that expand), expand, publish.
-        auto process = [&](const Cur& x, const uint32_t (&cv)[2][NL], const float (&av)[NS]) -> bool {
+        auto process = [&](const Cur& x, const uint32_t (&cv)[2][NL], const float (&av)[NSC]) -> bool {
             if (wl == 0) wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 9, 256u);  // a timeout shows in the abort flag
             ptx::named_bar_sync(kPfGroupBar0 + group, kPfGroupWarps * 32);
             if (*ctl.abort_flag) return false;
             const uint32_t line = smem_base + (uint32_t)s * kABytes + line_off;
-            float a2[NS];  // scales of the second 32 weights when they belong to the next group
+            float a2[NSC];  // scales of the second 32 weights when they belong to the next group
             if (x.split) {
                 const float* ap = alpha_ptr(x, x.c + 1);
 #pragma unroll
-                for (int i = 0; i < NS; ++i)
+                for (int i = 0; i < NSC; ++i)
                     a2[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
             }
 #pragma unroll
@@ -896,7 +896,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     uint32_t w8[BCQ_MAX_Q];
 #pragma unroll
                     for (int i = 0; i < BCQ_MAX_Q; ++i) {
-                        a8[i] = (second ? a2[i % NS] : av[i % NS]) * wscale;
+                        a8[i] = (second ? a2[i % NSC] : av[i % NSC]) * wscale;
                         w8[i] = cv[b][i % NL];
                     }
                     expand16_sum(w8, a8, p.q, line, lx, 4 * b);
@@ -907,7 +907,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                     if ((b == 0 && x.fresh) || second) {
                         float a[4];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) a[i] = (second ? a2[i % NS] : av[i % NS]) * wscale;
+                        for (int i = 0; i < 4; ++i) a[i] = (second ? a2[i % NSC] : av[i % NSC]) * wscale;
                         lut = (QM == QM_LUT4) ? build_lut(a[0], a[1], a[2], a[3]) : build_lut(a[0], a[1], a[2], 0.0f);
                     }
                     uint32_t cw[NWC], S[4];
@@ -943,7 +943,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             if (cur.valid) locate(cur);
         }
         uint32_t cvA[2][NL], cvB[2][NL];
-        float avA[NS], avB[NS];
+        float avA[NSC], avB[NSC];
         if (QM == QM_GENERIC) {
             // q > 4: one set of registers, loaded at the head of the task (under the wait for the slot)
             while (cur.valid && ok) {
@@ -1445,7 +1445,7 @@ struct ExpandPlan {
     int ld_act;                                                          // pitch of the fp16 activations (elements)
 };
 
-constexpr int kPfMinWidth = 176;                                       // token-tile width below which the workers, not the UMMAs, set the pace
+constexpr int kPfStageFixed = 224;                                     // fixed cost of a pipeline stage, in token-tile columns
 constexpr size_t kSmemLimit = 232448;                                   // 227 KiB per CTA
 constexpr size_t kPfFixedBytes = 1024 + kPfCtlBytes + kPfScaleBytes;   // alignment slack, barriers, output scales
 
@@ -1465,16 +1465,20 @@ ExpandPlan plan_expand(int mode, int d_out, int d_in, int q, int g, int n) {
     else if (n <= 64) tn = 64;
     else if (n <= 128) tn = 128;
     else {
-        // Any multiple of 16 up to 256 is a legal UMMA width.  The kernel is persistent with
-        // ceil(tiles / SMs) tiles per CTA, so its time goes with that count times the width (the
-        // UMMAs of a stage take time in proportion to it) -- except that below kPfMinWidth the
-        // workers, who expand one weight tile per stage whatever the width, set the pace.  The
-        // width that minimises the product wins; ties go to the wider tile (fewer expansions).
+        // Any multiple of 16 up to 256 is a legal UMMA width.  A stage of the kernel takes a fixed
+        // time (barriers, UMMA issue, the expansion of one weight tile whatever the width) plus a
+        // time in proportion to the width (the UMMAs themselves); measured, the fixed part is worth
+        // about kPfStageFixed columns.  The kernel is persistent with ceil(tiles / SMs) tiles per
+        // CTA, so a narrower tile can shorten the call (fewer tiles per CTA, less padding past n)
+        // but costs SM time that kernels running beside this one would have used.  The width
+        // that minimises call time x SM time wins; ties go to the wider tile.
         long long best = -1;
         tn = 256;
         for (int c = 256; c >= 128; c -= 16) {
-            const long long per_cta = ceil_div(pl.m_tiles * ceil_div(n, c), sms);
-            const long long cost = per_cta * (c > kPfMinWidth ? c : kPfMinWidth);
+            const long long tiles = (long long)pl.m_tiles * ceil_div(n, c);
+            const long long per_cta = (tiles + sms - 1) / sms;
+            const long long stage = c + kPfStageFixed;
+            const long long cost = (per_cta * stage) * (tiles * stage);
             if (best < 0 || cost < best) { best = cost; tn = c; }
         }
     }
