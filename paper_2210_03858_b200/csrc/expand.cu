@@ -425,7 +425,15 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
 #pragma unroll
         for (int i = 0; i < VPL; ++i) m = max(m, max_mag_bf16x8(held[i], (lane + 32 * i) * 8, p.K));
     } else {
-        for (int v = lane; v < nvec; v += 32) m = max(m, max_mag_bf16x8(__ldg(src + v), v * 8, p.K));
+        // long rows: four loads of a lane in flight at a time
+        for (int v0 = lane; v0 < nvec; v0 += 128) {
+            uint4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                x[u] = (v0 + 32 * u < nvec) ? __ldg(src + v0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) m = max(m, max_mag_bf16x8(x[u], (v0 + 32 * u) * 8, p.K));
+        }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -439,7 +447,15 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
             if (v < nvec) dst[v] = scale_to_fp16x8(held[i], v * 8, p.K, scale);
         }
     } else {
-        for (int v = lane; v < nvec; v += 32) dst[v] = scale_to_fp16x8(__ldg(src + v), v * 8, p.K, scale);
+        for (int v0 = lane; v0 < nvec; v0 += 128) {
+            uint4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                x[u] = (v0 + 32 * u < nvec) ? __ldg(src + v0 + 32 * u) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (v0 + 32 * u < nvec) dst[v0 + 32 * u] = scale_to_fp16x8(x[u], (v0 + 32 * u) * 8, p.K, scale);
+        }
     }
 }
 
@@ -1646,10 +1662,11 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     pp.act_blocks = tok_blocks;
     const unsigned pgrid = (unsigned)(tok_blocks + ablocks + pp.bits_blocks + alpha_tr_blocks);
     const int nvec = (Kdim + 7) / 8;
-    // Rows of up to 1024 elements stay in registers between the two passes over them.  Longer
+    // Rows of up to 2048 elements stay in registers between the two passes over them.  Longer
     // rows are read twice instead (the second time from L2): holding them would cost so many
     // registers that the grid no longer fits on the SMs in one wave.
     if (nvec <= 32 * 4) prepare_kernel<4><<<pgrid, 256, 0, s>>>(pp);
+    else if (nvec <= 32 * 8) prepare_kernel<8><<<pgrid, 256, 0, s>>>(pp);
     else prepare_kernel<0><<<pgrid, 256, 0, s>>>(pp);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
