@@ -174,7 +174,9 @@ bcq_status bcq_linear_decode(int d_out, int d_in, int q, int g, int n, const voi
  *     12288-row layer; 8 tokens of it fit).  Such problems need bcq_linear_decode.
  *   - The first call on each device looks up the device address of the array
  *     (cudaGetSymbolAddress) with that device current; make that first call outside any stream
- *     capture.  Later calls on the device only launch kernels.
+ *     capture.  Later calls on the device only launch kernels.  The address is kept for the
+ *     life of the process: after cudaDeviceReset on that device it is stale and the library
+ *     must be loaded again.
  *   - All calls on a device share the one array.  It keeps whatever the last call left in it;
  *     every call overwrites the part it reads, so nothing has to be cleared.  Two calls that may
  *     overlap on the GPU (different streams, no dependency) race on it: serialise them. */
@@ -282,6 +284,11 @@ unsigned long long bcq_kernel_launches(void);
 /* Reads (and with reset != 0 clears) the device-side flag that kernels set when a bounded wait
  * expired.  Synchronises the device.  *flag_out = 0 means no kernel has given up. */
 bcq_status bcq_device_timeout_flag(int* flag_out /* host */, int reset);
+/* Synchronises the device and reports its state as a status: BCQ_ERR_DEVICE_TIMEOUT if a kernel
+ * of this library has given up on a wait since the flag was last cleared (the results of the
+ * calls since then are not to be trusted; bcq_device_timeout_flag tells which wait and clears the
+ * flag), BCQ_ERR_CUDA if the synchronisation itself failed, BCQ_OK otherwise. */
+bcq_status bcq_check_device(void);
 
 #ifdef __cplusplus
 }

@@ -27,7 +27,7 @@ SYMBOLS = ("bcq_pitch_words", "bcq_bits_bytes", "bcq_num_groups", "bcq_alpha_cou
            "bcq_kernel_launches", "bcq_linear_decode_noalloc", "bcq_decode_pack_bytes",
            "bcq_decode_pack", "bcq_linear_decode_packed", "bcq_lr_linear_decay", "bcq_alpha_adamw",
            "bcq_alpha_pack", "bcq_alpha_unpack", "bcq_prepared_bytes", "bcq_prepare_planes",
-           "bcq_linear_fwd_prepared", "bcq_linear_bwd_x_prepared")
+           "bcq_linear_fwd_prepared", "bcq_linear_bwd_x_prepared", "bcq_check_device")
 
 
 class BcqError(RuntimeError):
@@ -104,6 +104,8 @@ def lib() -> C.CDLL:
         l.bcq_last_cuda_error.argtypes = []
         l.bcq_kernel_launches.restype = C.c_ulonglong
         l.bcq_kernel_launches.argtypes = []
+        l.bcq_check_device.restype = i
+        l.bcq_check_device.argtypes = []
         l.bcq_device_timeout_flag.restype = i
         l.bcq_device_timeout_flag.argtypes = [C.POINTER(C.c_int), i]
         _lib = l
@@ -398,6 +400,11 @@ def alpha_unpack(packed, alpha_flat, segments: Segments):
 
 def kernel_launches() -> int:
     return int(lib().bcq_kernel_launches())
+
+
+def check_device() -> None:
+    """Synchronises; raises BcqError (status BCQ_ERR_DEVICE_TIMEOUT) if a kernel gave up on a wait."""
+    _check(lib().bcq_check_device(), "bcq_check_device")
 
 
 def device_timeout_flag(reset: bool = False) -> int:

@@ -81,6 +81,13 @@ extern "C" bcq_status bcq_device_timeout_flag(int* flag_out, int reset) {
     return BCQ_OK;
 }
 
+extern "C" bcq_status bcq_check_device(void) {
+    int flag = 0;
+    const bcq_status st = bcq_device_timeout_flag(&flag, 0);
+    if (st != BCQ_OK) return st;
+    return flag != 0 ? BCQ_ERR_DEVICE_TIMEOUT : BCQ_OK;
+}
+
 extern "C" size_t bcq_workspace_bytes(int op, int d_out, int d_in, int q, int g, int n) {
     if (bcq::check_shape(d_out, d_in, q, g) != BCQ_OK) return 0;
     if (op != BCQ_OP_QUANTIZE && n < 1) return 0;

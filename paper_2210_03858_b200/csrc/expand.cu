@@ -1567,6 +1567,13 @@ DecodePlan plan_decode(int d_out, int d_in, int n) {
     return pl;
 }
 
+template <int MODE>
+bcq_status ensure_expand_smem(int q, size_t smem) {
+    if (q <= 3) return ensure_dynamic_smem(expand_gemm_kernel<MODE, QM_LUT3>, smem);
+    if (q == 4) return ensure_dynamic_smem(expand_gemm_kernel<MODE, QM_LUT4>, smem);
+    return ensure_dynamic_smem(expand_gemm_kernel<MODE, QM_GENERIC>, smem);
+}
+
 template <int MODE, int QM>
 bcq_status launch_expand(const CUtensorMap& tm, const CUtensorMap& tmo, const ExpandParams& p, const ExpandPlan& pl,
                          cudaStream_t stream) {
@@ -1635,6 +1642,17 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     bcq_status st = make_tmap_16bit(&tm, act16, 1, pl.ld_act, n, (size_t)pl.ld_act, pl.TN);
     if (st != BCQ_OK) return st;
 
+    // everything that can fail is done before the first launch: the output tensor map and the
+    // shared-memory limits of the kernels this call may run
+    const bool fast_epi = (out_dtype == BCQ_BF16 && pl.splits == 1 && aligned16(out) && (ldo * 2) % 16 == 0 &&
+                           ldo >= (size_t)Mdim);
+    CUtensorMap tmo = tm;
+    if (fast_epi) {
+        st = make_tmap_out_bf16(&tmo, out, Mdim, n, ldo);
+        if (st != BCQ_OK) return st;
+    }
+    if ((st = ensure_expand_smem<MODE>(q, pl.smem)) != BCQ_OK) return st;
+
     PrepParams pp;
     pp.n = n; pp.K = Kdim; pp.act_blocks = n;
     pp.ld_in = (long long)ldact; pp.ld_out = pl.ld_act;
@@ -1686,12 +1704,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     p.out = out; p.ldo = (long long)ldo; p.out_bf16 = (out_dtype == BCQ_BF16);
     p.partial = reinterpret_cast<float*>(wsb + pl.off_partial);
     // bf16 output with an aligned base and pitch and no K split goes out through TMA stores
-    CUtensorMap tmo = tm;
-    p.fast_epi = (p.out_bf16 && pl.splits == 1 && aligned16(out) && (ldo * 2) % 16 == 0 && ldo >= (size_t)Mdim) ? 1 : 0;
-    if (p.fast_epi) {
-        st = make_tmap_out_bf16(&tmo, out, Mdim, n, ldo);
-        if (st != BCQ_OK) return st;
-    }
+    p.fast_epi = fast_epi ? 1 : 0;
     // The workers find the last tile's accumulator by barrier parity alone.  They run at most
     // `a_slots` pipeline stages ahead of the tensor core, so the parity is unambiguous only if
     // two tiles are longer than that: then the accumulator's previous use (two tiles back) is
@@ -1759,9 +1772,9 @@ bcq_status run_decode(int d_out, int d_in, int q, int g, int n, const void* X, s
     return BCQ_OK;
 }
 
-bcq_status fwd_common(int decode, int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
-                      const uint32_t* bits, const float* alpha, const float* bias, void* Y, size_t ldy,
-                      int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+// Argument checks of the forward and decode entry points (host arithmetic and pointer tests only).
+bcq_status check_fwd_args(int decode, int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                          const uint32_t* bits, const float* alpha, const void* Y, size_t ldy, int y_dtype) {
     bcq_status st = check_shape(d_out, d_in, q, g);
     if (st != BCQ_OK) return st;
     if (n < 1 || (decode && n > 16)) return BCQ_ERR_SHAPE;
@@ -1770,6 +1783,14 @@ bcq_status fwd_common(int decode, int d_out, int d_in, int q, int g, int n, cons
     if (ldy < (size_t)d_out) return BCQ_ERR_SHAPE;
     if (y_dtype != BCQ_F32 && y_dtype != BCQ_BF16) return BCQ_ERR_SHAPE;
     if (!aligned16(bits)) return BCQ_ERR_ALIGN;
+    return BCQ_OK;
+}
+
+bcq_status fwd_common(int decode, int d_out, int d_in, int q, int g, int n, const void* X, size_t ldx,
+                      const uint32_t* bits, const float* alpha, const float* bias, void* Y, size_t ldy,
+                      int y_dtype, void* ws, size_t ws_bytes, void* stream) {
+    const bcq_status st = check_fwd_args(decode, d_out, d_in, q, g, n, X, ldx, bits, alpha, Y, ldy, y_dtype);
+    if (st != BCQ_OK) return st;
     if (decode)
         return run_decode(d_out, d_in, q, g, n, X, ldx, bits, alpha, bias, Y, ldy, y_dtype, ws, ws_bytes, stream);
     return run_expand<MODE_FWD>(d_out, d_in, q, g, n, X, ldx, bits, nullptr, alpha, bias, Y, ldy, y_dtype, ws,
@@ -1849,10 +1870,12 @@ extern "C" bcq_status bcq_linear_decode_noalloc(int d_out, int d_in, int q, int 
                                                 size_t ldx, const uint32_t* bits, const float* alpha,
                                                 const float* bias, void* Y, size_t ldy, int y_dtype,
                                                 void* stream) {
-    // validate first, so that a bad call neither touches the device nor resolves the symbol
-    bcq_status st = check_shape(d_out, d_in, q, g);
+    // Every argument is checked before the scratch symbol is resolved.  (The size check asks the
+    // device for its SM count, so it is not free of CUDA calls; without a device the count falls
+    // back to a B200's.)  The address found for a device is kept for the life of the process: after
+    // cudaDeviceReset it is stale, and the library has to be loaded again.
+    bcq_status st = check_fwd_args(1, d_out, d_in, q, g, n, X, ldx, bits, alpha, Y, ldy, y_dtype);
     if (st != BCQ_OK) return st;
-    if (n < 1 || n > 16) return BCQ_ERR_SHAPE;
     if (bcq::decode_workspace_bytes(d_out, d_in, q, g, n) > (size_t)BCQ_NOALLOC_SCRATCH_BYTES)
         return BCQ_ERR_WORKSPACE;
     void* scratch = nullptr;

@@ -29,6 +29,7 @@ def _built():
     bcq_build.build_library()
     assert torch.cuda.is_available()
     yield
+    bcq.check_device()  # raises if a kernel reported an expired wait
     assert bcq.device_timeout_flag() == 0, "a kernel reported an expired wait"
 
 
@@ -74,6 +75,8 @@ QUANT_CASES = [
     (16, 1024, 3, 1024, 3, 0.0),
     (6, 2304, 4, 2304, 2, 0.0),
     (12, 200, 5, 200, 1, 0.0),
+    (32, 768, 3, 128, 15, 1e-3),      # the 15 alternating rounds of the paper's appendix
+    (32, 768, 4, 128, 15, 1e-3),
 ]
 
 
