@@ -1680,11 +1680,11 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     pp.act_blocks = tok_blocks;
     const unsigned pgrid = (unsigned)(tok_blocks + ablocks + pp.bits_blocks + alpha_tr_blocks);
     const int nvec = (Kdim + 7) / 8;
-    // Rows of up to 2048 elements stay in registers between the two passes over them.  Longer
-    // rows are read twice instead (the second time from L2): holding them would cost so many
-    // registers that the grid no longer fits on the SMs in one wave.
+    // Rows of up to 1024 elements stay in registers between the two passes over them.  Longer
+    // rows are read twice instead (the second time from L2), four loads of a lane at a time:
+    // holding them costs so many registers that the blocks resident on an SM are too few to
+    // cover the memory latency (measured: 14.8 us against 11.3 us for 4096 rows of 1600).
     if (nvec <= 32 * 4) prepare_kernel<4><<<pgrid, 256, 0, s>>>(pp);
-    else if (nvec <= 32 * 8) prepare_kernel<8><<<pgrid, 256, 0, s>>>(pp);
     else prepare_kernel<0><<<pgrid, 256, 0, s>>>(pp);
     bcq::count_launch();
     BCQ_CUDA_TRY(cudaGetLastError());
