@@ -811,6 +811,8 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         struct Cur {
             int tile, it, iters, kb_begin, mt;
             int c, kpos, next_edge;  // group index of the task's first 32 k (forward: advances with the stage)
+            uint32_t code_idx;       // this thread's first word of the task in the regrouped planes
+            uint32_t alpha_idx;      // its first scale (plane 0, group c) in the regrouped scales
             bool split;              // the second 32 k belong to the next group (g not a multiple of 64)
             bool fresh;              // the scales differ from the previous task's: load them, rebuild the table
             bool valid;
@@ -820,11 +822,16 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             tile_coords(x.tile, m0, t0, z, x.kb_begin, x.iters);
             x.mt = m0 >> 7;
         };
-        auto locate = [&](Cur& x) {  // group index at (tile, it), from scratch
+        const uint32_t code_step = kPfGroups * chunk_words;
+        const uint32_t alpha_step = kPfGroups * (uint32_t)p.G * alpha_block;  // dX: the next task's rows
+        auto locate = [&](Cur& x) {  // group index and array positions at (tile, it), from scratch
             x.kpos = (MODE == MODE_FWD) ? (x.kb_begin + x.it) * kBlockK : x.mt * kBlockM + half * 64;
             x.c = min(x.kpos / p.g, p.G - 1);
             x.next_edge = (x.c + 1) * p.g;
             x.split = (x.kpos + 32 >= x.next_edge) && (x.c < p.G - 1);
+            x.code_idx = (uint32_t)(x.mt * p.num_kb + x.kb_begin + x.it) * chunk_words + word_off;
+            const int blk = (MODE == MODE_FWD) ? x.mt : x.kb_begin + x.it;
+            x.alpha_idx = (uint32_t)(blk * p.G + x.c) * alpha_block + (uint32_t)row;
         };
         // to the next task: kPfGroups stages on
         auto advance = [&](Cur& x) {
@@ -846,17 +853,17 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 while (x.kpos >= x.next_edge && x.c < p.G - 1) { ++x.c; x.next_edge += p.g; }
                 x.split = (x.kpos + 32 >= x.next_edge) && (x.c < p.G - 1);
                 x.fresh = (QM == QM_GENERIC) || (x.c != c0) || x.split;
+                x.code_idx += code_step;
+                x.alpha_idx += (uint32_t)(x.c - c0) * alpha_block;
             } else {
                 x.fresh = true;  // dX: every stage brings other rows
+                x.code_idx += code_step;
+                x.alpha_idx += alpha_step;
             }
-        };
-        auto alpha_ptr = [&](const Cur& x, int c) {
-            const int blk = (MODE == MODE_FWD) ? x.mt : x.kb_begin + x.it;
-            return p.alpha_t + ((long long)blk * p.G + c) * alpha_block + row;
         };
         // global loads of a task: its plane words or codes and, when they change, its scales
         auto issue = [&](const Cur& x, uint32_t (&cv)[2][NL], float (&av)[NSC]) {
-            const uint32_t* src = p.bits_t + ((long long)x.mt * p.num_kb + x.kb_begin + x.it) * chunk_words + word_off;
+            const uint32_t* src = p.bits_t + x.code_idx;
             if (QM == QM_GENERIC) {
 #pragma unroll
                 for (int i = 0; i < NL; ++i) {
@@ -878,7 +885,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
                 cv[1][0] = v1.y; cv[1][1] = v2.x; cv[1][2] = v2.y;
             }
             if (x.fresh) {
-                const float* ap = alpha_ptr(x, x.c);
+                const float* ap = p.alpha_t + x.alpha_idx;
 #pragma unroll
                 for (int i = 0; i < NSC; ++i)
                     av[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
@@ -899,7 +906,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const uint32_t line = smem_base + (uint32_t)s * kABytes + line_off;
             float a2[NSC];  // scales of the second 32 weights when they belong to the next group
             if (x.split) {
-                const float* ap = alpha_ptr(x, x.c + 1);
+                const float* ap = p.alpha_t + x.alpha_idx + alpha_block;  // group c + 1
 #pragma unroll
                 for (int i = 0; i < NSC; ++i)
                     a2[i] = (i < p.q) ? __uint_as_float(ptx::ldg_nc_u32(ap + i * kRows)) : 0.0f;
@@ -948,6 +955,7 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
         cur.split = false;
         cur.it = group;
         cur.iters = 0; cur.kb_begin = 0; cur.mt = 0; cur.c = 0; cur.kpos = 0; cur.next_edge = 0;
+        cur.code_idx = 0; cur.alpha_idx = 0;
         if (cur.valid) {
             enter_tile(cur);
             while (cur.it >= cur.iters) {
@@ -1628,6 +1636,8 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     const int Mdim = (MODE == MODE_FWD) ? d_out : d_in;
     const int Kdim = (MODE == MODE_FWD) ? d_in : d_out;
     const ExpandPlan pl = plan_expand(MODE, d_out, d_in, q, g, n);
+    // the kernel indexes the regrouped planes and scales with 32-bit word offsets
+    if ((pl.planes_bytes >> 2) >= (1ull << 32) || (pl.off_bits - pl.off_alpha) / 4 >= (1ull << 32)) return BCQ_ERR_UNSUPPORTED;
     if (ws == nullptr) return BCQ_ERR_NULL;
     if (ws_bytes < pl.total) return BCQ_ERR_WORKSPACE;
     if (!aligned16(ws)) return BCQ_ERR_ALIGN;
