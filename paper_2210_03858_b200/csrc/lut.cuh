@@ -133,10 +133,12 @@ __device__ __forceinline__ void selectors(const uint32_t (&v)[Q], uint32_t (&S)[
 }
 
 // 32 weights of one row: selector word r gives the eight fp16 values of 16-byte chunk chunk0 + r
-// of the row's 128-byte line (swizzle key lx), in natural k order.
+// of the row's 128-byte line (swizzle key lx), in natural k order.  `line` is 128-byte aligned, so
+// the swizzled chunk address is line ^ (lx << 4) ^ (chunk << 4): one XOR per store.
 template <int Q>
 __device__ __forceinline__ void expand32_codes(const uint32_t (&S)[4], const Lut& t, uint32_t line, uint32_t lx,
                                                uint32_t chunk0) {
+    const uint32_t linex = line ^ (lx << 4);
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
         // (shifts written as multiplications run on the multiply-add pipe; the logic pipe, which does
@@ -152,7 +154,7 @@ __device__ __forceinline__ void expand32_codes(const uint32_t (&S)[4], const Lut
             hbl ^= prmt(fa, S[r], 0xD9C8u) & 0x80808080u;
             hbh ^= prmt(fa, S[r], 0xFBEAu) & 0x80808080u;
         }
-        ptx::st_shared_v4(line + (((chunk0 + r) ^ lx) << 4), prmt(lbl, hbl, 0x5140u), prmt(lbl, hbl, 0x7362u),
+        ptx::st_shared_v4(linex ^ ((chunk0 + r) << 4), prmt(lbl, hbl, 0x5140u), prmt(lbl, hbl, 0x7362u),
                           prmt(lbh, hbh, 0x5140u), prmt(lbh, hbh, 0x7362u));
     }
 }
