@@ -263,7 +263,9 @@ class Stack:
 
     def per_op(self, main):
         """GPU time of each operation alone: its calls back to back on one stream (a graph, so
-        host launch time stays out), best of three."""
+        host launch time stays out).  Three untimed replays bring the clocks to where they settle
+        under load, then five replays are timed as one region and averaged: a single replay after an
+        idle gap runs at boost clocks and its time moves by tens of percent from run to run."""
         torch = self.torch
         res = {}
         for name in self.OPS:
@@ -271,16 +273,16 @@ class Stack:
             with torch.cuda.graph(g_, stream=main):
                 for l in self.layers:
                     self.op(name, l)
-            g_.replay()
-            torch.cuda.synchronize()
-            best = None
             for _ in range(3):
-                a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
                 g_.replay()
-                b_.record()
-                torch.cuda.synchronize()
-                best = a.elapsed_time(b_) if best is None else min(best, a.elapsed_time(b_))
+            torch.cuda.synchronize()
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(5):
+                g_.replay()
+            b_.record()
+            torch.cuda.synchronize()
+            best = a.elapsed_time(b_) / 5.0
             flops = sum(2.0 * self.cfg["tokens"] * l["d_in"] * l["d_out"] for l in self.layers)
             res[name] = (best, flops, len(self.layers))
             del g_
