@@ -52,7 +52,6 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
               const DalphaParams p) {
     constexpr uint32_t kBBytes = TN * kBlockK * 2;
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
-    constexpr uint32_t kIdesc = ptx::make_idesc_bf16(kBlockM, TN, 1, 1);
     constexpr int HN = TN / 2;
     constexpr int NCH = HN / 32;
     constexpr uint32_t kAccCols = TmemCols<TN>::value;
@@ -121,18 +120,21 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 int j0, k0, z, kb_begin, iters;
                 tile_coords(tile, j0, k0, z, kb_begin, iters);
+                // a column tile that reaches past d_in brings (and multiplies) only the 64-column
+                // blocks that hold columns of the matrix
+                const int boxes = min(TN / 64, (p.d_in - k0 + 63) / 64);
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.empty + 8 * s, ph ^ 1u, ctl, 11);
                     if (!ok) break;
                     const uint32_t sa = smem_base + s * kStageBytes;
                     const int tok = (kb_begin + it) * kBlockK;
-                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kStageBytes);
+                    ptx::mbar_arrive_expect_tx(ctl.full + 8 * s, kABytes + (uint32_t)boxes * 8192u);
                     // A: two blocks of 64 rows j (inner) x 64 tokens; B: TN/64 blocks of 64 k x 64 tokens
                     ptx::tma_load_2d(sa, &tmap_dy, j0, tok, ctl.full + 8 * s);
                     ptx::tma_load_2d(sa + 8192, &tmap_dy, j0 + 64, tok, ctl.full + 8 * s);
 #pragma unroll
                     for (int b = 0; b < TN / 64; ++b)
-                        ptx::tma_load_2d(sa + kABytes + b * 8192, &tmap_x, k0 + b * 64, tok, ctl.full + 8 * s);
+                        if (b < boxes) ptx::tma_load_2d(sa + kABytes + b * 8192, &tmap_x, k0 + b * 64, tok, ctl.full + 8 * s);
                     in_flight = min(in_flight + 1, STAGES);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
@@ -167,6 +169,8 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)acc * kAccCols;
+                const int boxes = min(TN / 64, (p.d_in - k0 + 63) / 64);
+                const uint32_t idesc = ptx::make_idesc_bf16(kBlockM, boxes * 64, 1, 1);  // the UMMA is as wide as the tile's columns
                 for (int it = 0; it < iters; ++it) {
                     ok = wait_bar(ctl.full + 8 * s, ph, ctl, 13, 32u);
                     if (!ok) break;
@@ -175,7 +179,7 @@ dalpha_kernel(const __grid_constant__ CUtensorMap tmap_dy, const __grid_constant
                     const uint32_t b_lo = a_lo + (kABytes >> 4);
 #pragma unroll
                     for (int kk = 0; kk < kBlockK / 16; ++kk)
-                        ptx::umma_f16_halves(d_tmem, a_lo + kk * (2048u >> 4), kHi, b_lo + kk * (2048u >> 4), kHi, kIdesc,
+                        ptx::umma_f16_halves(d_tmem, a_lo + kk * (2048u >> 4), kHi, b_lo + kk * (2048u >> 4), kHi, idesc,
                                              (it > 0 || kk > 0) ? 1u : 0u);
                     ptx::umma_commit(ctl.empty + 8 * s);
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
