@@ -1052,9 +1052,11 @@ expand_gemm_kernel(const __grid_constant__ CUtensorMap tmap_b, const __grid_cons
             const uint32_t acc_ph = (lt >> 1) & 1;
             for (int i = et; i < TN; i += kPfEpiWarps * 32)
                 scale[i] = (t0 + i < p.n) ? winv * __ldg(p.tok_inv_scale + t0 + i) : 0.0f;
+            // one warp polls the accumulator's barrier (a whole tile away), the others park on the
+            // hardware barrier that also publishes the scale row; a timeout shows in the abort flag
+            if (ew == 0) wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7, 1000u);
             asm volatile("bar.sync 2, %0;" ::"n"(kPfEpiWarps * 32) : "memory");
-            ok = wait_bar(ctl.accum + 8 * acc, acc_ph, ctl, 7, 1000u);  // a whole tile away: poll rarely
-            if (!ok) break;
+            if (*ctl.abort_flag) { ok = false; break; }
             ptx::tc_fence_after_sync();
             // accumulator row `lane` of this warp's quarter is output column m0w + lrow
             const int m0w = m0 + quarter * 32;
