@@ -247,6 +247,20 @@ def test_prepared_planes_need_at_most_four_planes():
 
 # --------------------------------------------------------------------------- tile-schedule corners
 
+@pytest.mark.parametrize("n", [129, 145, 257, 300, 530, 1000])
+def test_fwd_and_bwd_x_with_token_counts_between_tile_widths(n):
+    # above 128 tokens the token-tile width is any multiple of 16 up to 256, chosen per call: these
+    # counts give widths that are not powers of two, ragged last tiles and single tiles wider than n
+    d_in, d_out, q, g = 640, 2560, 4, 128
+    _, X, dY, bits, alpha, _, _ = make_case(900 + n, n, d_in, d_out, q, g)
+    Xd, dYd, bd, ad = _upload(X, dY, bits, alpha)
+    ref_y = oracle.fwd(X, bits, alpha, d_in, g)
+    ref_dx = oracle.bwd_x(dY, bits, alpha, d_in, g)
+    for dt, tol in ((torch.float32, TOL), (torch.bfloat16, TOL + 2.0 ** -8)):
+        assert rel_err(bcq.linear_fwd(Xd, bd, ad, d_in, g, out_dtype=dt).float().cpu().numpy(), ref_y) <= tol
+        assert rel_err(bcq.linear_bwd_x(dYd, bd, ad, d_in, g, out_dtype=dt).float().cpu().numpy(), ref_dx) <= tol
+
+
 @pytest.mark.parametrize("n", [1, 17, 31, 32])
 def test_fwd_and_bwd_x_with_few_tokens(n):
     # the prefill entry points accept any n >= 1; n <= 32 takes the narrowest token tile
