@@ -292,6 +292,13 @@ struct PrepParams {
 constexpr int kPrepTokensPerBlock = 8;
 
 __device__ __forceinline__ uint32_t max_mag_bf16x8(const uint4& x, int k0, int K) {
+    if (k0 + 8 <= K) {
+        // whole vector inside the row: magnitudes are 15-bit integers, compared two per word
+        const uint32_t a = __vmaxu2(x.x & 0x7FFF7FFFu, x.y & 0x7FFF7FFFu);
+        const uint32_t b = __vmaxu2(x.z & 0x7FFF7FFFu, x.w & 0x7FFF7FFFu);
+        const uint32_t c = __vmaxu2(a, b);
+        return max(c & 0xFFFFu, c >> 16);
+    }
     const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
     uint32_t m = 0u;
 #pragma unroll
@@ -302,6 +309,16 @@ __device__ __forceinline__ uint32_t max_mag_bf16x8(const uint4& x, int k0, int K
 
 __device__ __forceinline__ uint4 scale_to_fp16x8(const uint4& x, int k0, int K, float scale) {
     const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    if (k0 + 8 <= K) {
+        // bf16 -> fp32 is a shift (low half) or a mask (high half); the product with a power of two
+        // is exact and one conversion packs two of them
+        uint4 o;
+        uint32_t* ow = &o.x;
+#pragma unroll
+        for (int w = 0; w < 4; ++w)
+            ow[w] = pack_half2(__uint_as_float(xs[w] << 16) * scale, __uint_as_float(xs[w] & 0xFFFF0000u) * scale);
+        return o;
+    }
     float f[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
