@@ -348,6 +348,30 @@ __global__ void __launch_bounds__(256) prepare_kernel(const PrepParams p) {
         int b = bid - p.act_blocks - p.amax_blocks;
         const bool is_alpha = b >= p.bits_blocks;
         if (is_alpha) b -= p.bits_blocks;
+        if (is_alpha) {
+            // ---- scales of one plane and one tile of 128 rows: alpha[i][j][c] is contiguous over
+            // (j, c), so the block reads it as one coalesced run and scatters the values to their
+            // places in the regrouped array (rows past d_out become zeros)
+            const int rt = b % p.row_tiles;
+            const int i = b / p.row_tiles;
+            const float* src = p.alpha + ((long long)i * p.d_out + (long long)rt * 128) * p.G;
+            const int count = 128 * p.G;
+            const int rows_left = p.d_out - rt * 128;
+            for (int e = threadIdx.x; e < count; e += 256) {
+                const int r = e / p.G, c = e - r * p.G;
+                const float v = (r < rows_left) ? __ldg(src + e) : 0.0f;
+                long long o;
+                if (p.mode == MODE_FWD) {
+                    o = (((long long)rt * p.G + c) * p.q + i) * 128 + r;
+                } else {
+                    const int jb = rt * 2 + (r >> 6), rr = r & 63;
+                    if (jb >= p.num_kb) continue;
+                    o = (((long long)jb * p.G + c) * p.q + i) * 64 + rr;
+                }
+                p.alpha_t[o] = v;
+            }
+            return;
+        }
         const int cblks = is_alpha ? p.alpha_cblk : p.bits_cblk;
         const int cb = b % cblks;
         const int rt = (b / cblks) % p.row_tiles;
@@ -1698,7 +1722,7 @@ bcq_status run_expand(int d_out, int d_in, int q, int g, int n, const void* act,
     pp.alpha_cblk = ceil_div(pp.G, 32);
     const bool coded = q <= 4;  // selector codes (written once, or by the launch below); q > 4: plane words
     pp.bits_blocks = coded ? 0 : q * pp.row_tiles * pp.bits_cblk;
-    const int alpha_tr_blocks = q * pp.row_tiles * pp.alpha_cblk;
+    const int alpha_tr_blocks = q * pp.row_tiles;  // one block per (plane, tile of 128 rows)
     pp.bits = bits;
     pp.alpha_t = reinterpret_cast<float*>(wsb + pl.off_alpha);
     pp.bits_t = reinterpret_cast<uint32_t*>(wsb + pl.off_bits);
