@@ -84,9 +84,60 @@ __device__ bool solve_ls(int q, double m, double (*A)[BCQ_MAX_Q + 1], float* alp
     return true;
 }
 
-template <int EPT, int TW, bool ALT>
+// The same elimination for a plane count known at compile time: every index is static, so the
+// matrix stays in registers (the pivot row is found by value and swapped in by predicated moves).
+// Same operations in the same order as solve_ls, hence the same result.
+template <int Q>
+__device__ __forceinline__ bool solve_ls_static(double m, double (&A)[Q][Q + 1], float (&alpha)[Q]) {
+    const double tiny = 1e-12 * m;
+#pragma unroll
+    for (int col = 0; col < Q; ++col) {
+        int piv = col;
+        double best = fabs(A[col][col]);
+#pragma unroll
+        for (int r = col + 1; r < Q; ++r) {
+            const double v = fabs(A[r][col]);
+            if (v > best) { best = v; piv = r; }
+        }
+        if (best < tiny) return false;
+#pragma unroll
+        for (int r = col + 1; r < Q; ++r) {
+            if (r == piv) {
+#pragma unroll
+                for (int l = 0; l <= Q; ++l) {
+                    const double tmp = A[col][l];
+                    A[col][l] = A[r][l];
+                    A[r][l] = tmp;
+                }
+            }
+        }
+#pragma unroll
+        for (int r = col + 1; r < Q; ++r) {
+            const double f = __ddiv_rn(A[r][col], A[col][col]);
+#pragma unroll
+            for (int l = col; l <= Q; ++l) A[r][l] = __dsub_rn(A[r][l], __dmul_rn(f, A[col][l]));
+        }
+    }
+    double x[Q];
+#pragma unroll
+    for (int r = Q - 1; r >= 0; --r) {
+        double s = A[r][Q];
+#pragma unroll
+        for (int l = r + 1; l < Q; ++l) s = __dsub_rn(s, __dmul_rn(A[r][l], x[l]));
+        x[r] = __ddiv_rn(s, A[r][r]);
+    }
+#pragma unroll
+    for (int i = 0; i < Q; ++i) alpha[i] = (float)x[i];
+    return true;
+}
+
+// QT > 0: the number of planes as a compile-time constant (alternating path for q = 2, 3, 4: the
+// scales and the normal equations then live in registers); QT = 0: p.q at run time.
+template <int EPT, int TW, bool ALT, int QT>
 __global__ void __launch_bounds__(TW == 1 ? 128 : TW * 32)
 quantize_kernel(const QuantParams p) {
+    constexpr int QN = QT > 0 ? QT : BCQ_MAX_Q;
+    const int q = QT > 0 ? QT : p.q;
     constexpr int NT = TW * 32;
     constexpr int TEAMS = (TW == 1) ? 4 : 1;
     __shared__ double red_scratch[32];
@@ -124,9 +175,9 @@ quantize_kernel(const QuantParams p) {
             }
         }
 
-        float a[BCQ_MAX_Q];
-        // ---- greedy planes
-        for (int i = 0; i < p.q; ++i) {
+        float a[QN];
+        // ---- greedy planes (q is a constant for QT > 0: the loops over planes unroll by themselves)
+        for (int i = 0; i < q; ++i) {
             double local = 0.0;
 #pragma unroll
             for (int e = 0; e < EPT; ++e)
@@ -148,18 +199,18 @@ quantize_kernel(const QuantParams p) {
         }
 
         if (ALT) {
-            const int ncodes = 1 << p.q;
+            const int ncodes = 1 << q;
             for (int it = 0; it <= p.alt_iters; ++it) {
                 // ---- least-squares alpha for the current signs
-                double A[BCQ_MAX_Q][BCQ_MAX_Q + 1];
-                for (int i = 0; i < p.q; ++i) {
+                double A[QN][QN + 1];
+                for (int i = 0; i < q; ++i) {
                     double local = 0.0;
 #pragma unroll
                     for (int e = 0; e < EPT; ++e)
                         if (e * NT + tid < m) local += ((code[e] >> i) & 1u) ? (double)w[e] : -(double)w[e];
-                    A[i][p.q] = team_sum<TW>(local, red_scratch);
+                    A[i][q] = team_sum<TW>(local, red_scratch);
                     A[i][i] = md;
-                    for (int l = i + 1; l < p.q; ++l) {
+                    for (int l = i + 1; l < q; ++l) {
                         double cnt = 0.0;
 #pragma unroll
                         for (int e = 0; e < EPT; ++e)
@@ -169,13 +220,14 @@ quantize_kernel(const QuantParams p) {
                         A[l][i] = A[i][l];
                     }
                 }
-                solve_ls(p.q, md, A, a);
+                if constexpr (QT > 0) solve_ls_static<QT>(md, A, a);
+                else solve_ls(q, md, A, a);
                 if (it == p.alt_iters) break;  // the last pass is the final refit only
                 // ---- every weight moves to the nearest level; largest code wins ties
                 team_sync<TW>();
                 for (int s = tid; s < ncodes; s += NT) {
                     double L = 0.0;
-                    for (int i = 0; i < p.q; ++i) L = ((s >> i) & 1) ? L + (double)a[i] : L - (double)a[i];
+                    for (int i = 0; i < q; ++i) L = ((s >> i) & 1) ? L + (double)a[i] : L - (double)a[i];
                     levels[s] = L;
                 }
                 team_sync<TW>();
@@ -196,7 +248,7 @@ quantize_kernel(const QuantParams p) {
                 }
             }
             // ---- write the planes
-            for (int i = 0; i < p.q; ++i) {
+            for (int i = 0; i < q; ++i) {
                 uint32_t* brow = p.bits + ((long long)i * p.d_out + j) * p.pitch + (k0 >> 5);
 #pragma unroll
                 for (int e = 0; e < EPT; ++e) {
@@ -208,11 +260,17 @@ quantize_kernel(const QuantParams p) {
         }
 
         // ---- scales, zero padding words of the row, optional squared error
-        if (tid < p.q) p.alpha[((long long)tid * p.d_out + j) * p.G + c] = a[tid];
+        if constexpr (QT > 0) {
+#pragma unroll
+            for (int i = 0; i < QT; ++i)
+                if (tid == i) p.alpha[((long long)i * p.d_out + j) * p.G + c] = a[i];
+        } else {
+            if (tid < q) p.alpha[((long long)tid * p.d_out + j) * p.G + c] = a[tid];
+        }
         if (c == p.G - 1) {
             const int first_pad = (p.d_in + 31) >> 5;
             const int npad = p.pitch - first_pad;  // 0..3
-            for (int t = tid; t < npad * p.q; t += NT) {
+            for (int t = tid; t < npad * q; t += NT) {
                 const int i = t / npad, wdx = t - i * npad;
                 p.bits[((long long)i * p.d_out + j) * p.pitch + first_pad + wdx] = 0u;
             }
@@ -224,7 +282,7 @@ quantize_kernel(const QuantParams p) {
                 for (int e = 0; e < EPT; ++e)
                     if (e * NT + tid < m) {
                         double wh = 0.0;
-                        for (int i = 0; i < p.q; ++i)
+                        for (int i = 0; i < q; ++i)
                             wh = ((code[e] >> i) & 1u) ? wh + (double)a[i] : wh - (double)a[i];
                         const double d = (double)w[e] - wh;
                         local += d * d;
@@ -247,10 +305,14 @@ cudaError_t launch_quantize(const QuantParams& p, cudaStream_t stream) {
     long long blocks = (p.items + TEAMS - 1) / TEAMS;
     const long long cap = (long long)bcq::sm_count() * 64;  // grid-stride beyond this
     if (blocks > cap) blocks = cap;
-    if (p.alt_iters > 0)
-        quantize_kernel<EPT, TW, true><<<(unsigned)blocks, threads, 0, stream>>>(p);
-    else
-        quantize_kernel<EPT, TW, false><<<(unsigned)blocks, threads, 0, stream>>>(p);
+    if (p.alt_iters > 0) {
+        if (p.q == 2) quantize_kernel<EPT, TW, true, 2><<<(unsigned)blocks, threads, 0, stream>>>(p);
+        else if (p.q == 3) quantize_kernel<EPT, TW, true, 3><<<(unsigned)blocks, threads, 0, stream>>>(p);
+        else if (p.q == 4) quantize_kernel<EPT, TW, true, 4><<<(unsigned)blocks, threads, 0, stream>>>(p);
+        else quantize_kernel<EPT, TW, true, 0><<<(unsigned)blocks, threads, 0, stream>>>(p);
+    } else {
+        quantize_kernel<EPT, TW, false, 0><<<(unsigned)blocks, threads, 0, stream>>>(p);
+    }
     bcq::count_launch();
     return cudaGetLastError();
 }
