@@ -44,6 +44,14 @@ __device__ __forceinline__ double team_sum(double v, double* scratch) {
     return t;
 }
 
+// Sum of small non-negative counts over the team, as a double.  A warp adds them with one
+// integer reduction (exact, like the fp64 tree: the values are integers far below 2^53).
+template <int TW>
+__device__ __forceinline__ double team_count(int v, double* scratch) {
+    if (TW == 1) return (double)__reduce_add_sync(0xffffffffu, v);
+    return team_sum<TW>((double)v, scratch);
+}
+
 template <int TW>
 __device__ __forceinline__ void team_sync() {
     if (TW == 1)
@@ -211,11 +219,11 @@ quantize_kernel(const QuantParams p) {
                     A[i][q] = team_sum<TW>(local, red_scratch);
                     A[i][i] = md;
                     for (int l = i + 1; l < q; ++l) {
-                        double cnt = 0.0;
+                        int cnt = 0;
 #pragma unroll
                         for (int e = 0; e < EPT; ++e)
-                            if (e * NT + tid < m) cnt += (double)(((code[e] >> i) ^ (code[e] >> l)) & 1u);
-                        const double mism = team_sum<TW>(cnt, red_scratch);
+                            if (e * NT + tid < m) cnt += (int)(((code[e] >> i) ^ (code[e] >> l)) & 1u);
+                        const double mism = team_count<TW>(cnt, red_scratch);
                         A[i][l] = md - 2.0 * mism;
                         A[l][i] = A[i][l];
                     }
