@@ -167,6 +167,8 @@ quantize_kernel(const QuantParams p) {
         const int k0 = c * p.g;
         const int m = min(p.g, p.d_in - k0);
         const double md = (double)m;
+        const bool m_pow2 = (m & (m - 1)) == 0;
+        const double inv_m = 1.0 / md;
 
         double r[EPT];
         float w[ALT ? EPT : 1];
@@ -191,7 +193,8 @@ quantize_kernel(const QuantParams p) {
             for (int e = 0; e < EPT; ++e)
                 if (e * NT + tid < m) local += fabs(r[e]);
             const double S = team_sum<TW>(local, red_scratch);
-            a[i] = (float)__ddiv_rn(S, md);
+            // a power-of-two group size divides exactly by multiplying with its reciprocal
+            a[i] = (float)(m_pow2 ? __dmul_rn(S, inv_m) : __ddiv_rn(S, md));
             const double ad = (double)a[i];
             uint32_t* brow = p.bits + ((long long)i * p.d_out + j) * p.pitch + (k0 >> 5);
 #pragma unroll
